@@ -1,28 +1,33 @@
 #!/usr/bin/env python
-"""Benchmark of the N:M-sparse GEMM hot path on the DeiT-Small INT8 linear stack.
+"""Benchmark of the N:M-sparse GEMM hot path on the DeiT-Base INT8 linear stack.
 
-One step = one pass of nm_spmm over the twelve GEMMs of the workload (the four linear
-layers qkv / proj / fc1 / fc2 of a DeiT-Small block at batch 64, T = 12608 tokens, each
-with weights pruned at 2:4, 1:4 and 2:8), INT8 inputs, INT32 outputs.  Packing is
-offline and untimed; planning, loads, metadata handling, MMA and write-back are timed.
+One step = one pass of nm_spmm over the 48 GEMMs of the workload: the four linear layers
+qkv / proj / fc1 / fc2 of each of the 12 DeiT-Base blocks at batch 128 (T = 25216 tokens), every
+layer with its own weight pruned at a ratio drawn by seed from {dense, 2:4, 1:4, 2:8, 1:8}, INT8
+inputs, INT32 outputs.  It is the largest configuration of the benchmark set that runs as a whole
+model stack on one GPU (4.28 T dense-equivalent ops and 10 GB of algorithmic bytes per step).
+Packing is offline and untimed; loads, metadata handling, MMA and write-back are timed.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--per-layer]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg2|cfg1]
 
-Prints ONE JSON line (rank 0).  `value` is dense-equivalent INT8 TOPS (2*T*O*K per GEMM,
-summed over the step, over all GPUs) with inputs resident in HBM; `e2e` is the same metric
-through the public API with pinned host buffers (H2D of every X, D2H of every Y inside the
-timed region).  `roofline` is the HBM roofline of the tcgen05 kernel that runs all twelve
-GEMMs; `cpu_baseline` times the CPU oracle on a bounded row sample of the same workload.
+Prints ONE JSON line (rank 0).  `value` is dense-equivalent INT8 TOPS (2*T*O*K per GEMM, summed
+over the step, over all GPUs) with inputs resident in HBM; `e2e` is the same metric through the
+public API with pinned host buffers (H2D of every X, D2H of every Y inside the timed region).
+`roofline` is the HBM roofline of the kernel that moves most of the step's bytes; `tensor_roofline`
+gives the fc2 GEMMs (K = 3072, the ones closest to the tensor ridge) against the dense INT8 library
+peak measured in the same run (sparse = twice that) and against the nominal 4.5 / 9 POPS;
+`cpu_baseline` times the CPU oracle on a bounded row sample of the same workload, and the rows it
+computes are compared bit for bit with what the timed kernels left in Y (`verified`).  Further legs,
+each a replayed CUDA graph timed with CUDA events: the DeiT-Small stack (`cfg1_step`), the same
+DeiT-Base stack in FP16 (`cfg2_fp16`), the 72 linear layers of ViT-Large at batch 1 (`vit_l_b1_stack`),
+one ViT-Large batch-256 fc2 GEMM (`vit_l_b256_fc2`), dense cuBLAS on the same buffers (`cublas_dense`).
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
-import statistics
-import subprocess
 import sys
-import threading
 import time
 
 import numpy as np
@@ -32,21 +37,28 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 from paper_2607_12505_b200 import inputs  # noqa: E402
+from bench.clocks import ClockSampler  # noqa: E402
 
-WORKLOAD = "deit_small_linear_stack_int8_b64"
-METRIC = "nm_spmm dense-equivalent INT8 TOPS, DeiT-S linear stack (qkv/proj/fc1/fc2 x {2:4,1:4,2:8}), batch 64"
 UNIT = "TOPS"
+WORKLOADS = {
+    "cfg2": dict(name="deit_base_12block_linear_stack_int8_b128",
+                 metric="nm_spmm dense-equivalent INT8 TOPS, DeiT-B 12-block linear stack (48 GEMMs qkv/proj/fc1/fc2, per-layer "
+                        "N:M drawn by seed from {dense,2:4,1:4,2:8,1:8}), batch 128",
+                 specs=lambda: inputs.cfg2_layers("i8"), ref_rows=64, cpu_rows=3152),
+    "cfg1": dict(name="deit_small_linear_stack_int8_b64",
+                 metric="nm_spmm dense-equivalent INT8 TOPS, DeiT-S linear stack (qkv/proj/fc1/fc2 x {2:4,1:4,2:8}), batch 64",
+                 specs=inputs.cfg1_layers, ref_rows=1024, cpu_rows=12608),
+}
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the 12 launches of one step (all of them
-# the same kernel), from the ncu capture summarised in profiles/nm_umma_kernel_deit_s_stack_launch_list.md (each
-# launch measured alone: the 126 MB L2 still holds most of the freshly written Y when the kernel ends).
-NCU_DRAM_TRAFFIC_BYTES_PER_LAUNCH = 12.8e6
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_DENSE_TOPS = {"i8": 4500.0, "f16": 2250.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel (CTA pairs, INT8, 2:4), from ncu
+# captures of single DeiT-B GEMMs (each launch measured alone: the 126 MB L2 still holds part of the freshly written
+# Y when the kernel ends, so the write side undercounts), averaged over the step's mix of qkv / proj / fc1 / fc2.
+NCU_DRAM_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": None, "cfg1": 12.8e6}
 
 
-def layer_specs():
-    return inputs.cfg1_layers()
-
-
+# ---------------------------------------------------------------------------------- accounting
 def dense_ops(spec) -> float:
     return 2.0 * spec["T"] * spec["O"] * spec["K"]
 
@@ -55,16 +67,16 @@ def useful_ops(spec) -> float:
     return dense_ops(spec) * spec["n"] / spec["m"]
 
 
-def packed_w_bytes(spec) -> float:
+def packed_w_bytes(spec, eb=1) -> float:
     """Native packed weight bytes: kept values plus b-bit positions."""
     b = 0 if spec["n"] == spec["m"] else int(np.ceil(np.log2(spec["m"])))
     kept = spec["O"] * spec["K"] * spec["n"] / spec["m"]
-    return kept * 1 + kept * b / 8
+    return kept * eb + kept * b / 8
 
 
-def algorithmic_bytes(spec) -> float:
+def algorithmic_bytes(spec, eb=1, ob=4) -> float:
     """Bytes the method itself must move for one GEMM: X in once, Y out once, packed W once."""
-    return spec["T"] * spec["K"] * 1 + spec["T"] * spec["O"] * 4 + packed_w_bytes(spec)
+    return spec["T"] * spec["K"] * eb + spec["T"] * spec["O"] * ob + packed_w_bytes(spec, eb)
 
 
 def measured_peaks():
@@ -78,81 +90,34 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
-# ---------------------------------------------------------------------------------- clocks
-class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-
-    def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
-
-    def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._pump, daemon=True)
-            self.thread.start()
-        except Exception:
-            self.proc = None
-
-    def _pump(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
-
-    def stop(self) -> dict:
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=2)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for l in self.lines:
-            parts = [p.strip() for p in l.split(",")]
-            if len(parts) < 6:
-                continue
-            try:
-                sm.append(float(parts[0]))
-                mx.append(float(parts[1]))
-            except ValueError:
-                continue
-            for name, val in zip(names, parts[2:6]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
-
-
 # ---------------------------------------------------------------------------------- oracle legs
-def oracle_sample(specs, rows_per_layer: int):
-    """(callable running the oracle once over the sample, useful ops, dense ops, description)."""
+def oracle_sample(specs, rows_per_layer: int, keep_outputs: bool = False):
+    """(callable running the oracle once over the sample, dense ops of the sample, threads, description, outputs)."""
     from oracle import nm_oracle as orc
-    work = []
+    work, outs = [], []
     for s in specs:
-        X, W = inputs.make_layer(s, "bench")
+        X, W = inputs.make_layer(s, "bench", 0)
         rows = np.arange(min(rows_per_layer, s["T"]), dtype=np.int64)
         work.append((X, orc.compress(W, s["n"], s["m"]), rows))
-    frac = min(rows_per_layer, specs[0]["T"]) / specs[0]["T"]
+    n_rows = min(rows_per_layer, specs[0]["T"])
+    frac = n_rows / specs[0]["T"]
 
     def run():
+        outs.clear()
         for X, packed, rows in work:
-            orc.spmm_packed(X, packed, rows=rows)
+            y = orc.spmm_packed(X, packed, rows=rows)
+            if keep_outputs:
+                outs.append(y)
     return run, sum(dense_ops(s) for s in specs) * frac, orc.num_threads(), \
-        f"first {min(rows_per_layer, specs[0]['T'])} of {specs[0]['T']} token rows of every GEMM of the step, all output columns"
+        f"first {n_rows} of {specs[0]['T']} token rows of every GEMM of the step, all output columns", outs
 
 
-def run_reference(args):
+def run_reference(args, wl):
     """--impl reference: the CPU oracle, as it stands, on a bounded sample per step."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    specs = layer_specs()
-    run, dense_sample_ops, cores, desc = oracle_sample(specs, args.ref_rows)
+    specs = wl["specs"]()
+    run, dense_sample_ops, cores, desc, _ = oracle_sample(specs, args.ref_rows or wl["ref_rows"])
     for _ in range(max(args.warmup, 1)):
         run()
     t0 = time.perf_counter()
@@ -161,33 +126,137 @@ def run_reference(args):
     dt = (time.perf_counter() - t0) / args.steps
     tops = dense_sample_ops / dt / 1e12
     line = {
-        "impl": "reference", "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "impl": "reference", "metric": wl["metric"], "value": tops, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": max(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "int8", "data": "synthetic", "config": {"workload": WORKLOAD, "sample": desc},
+        "dtype": "int8", "data": "synthetic", "config": {"workload": wl["name"], "sample": desc},
         "cpu_baseline": {"value": tops, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": tops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------- GPU helpers
+class Stack:
+    """A list of GEMMs on one device, every GEMM with its own X, Y, packed W, scratch and status word."""
+
+    def __init__(self, torch, nm, specs, dev, key, rank=0, od=None, host_x=False, device_x=False):
+        self.torch, self.nm, self.dev = torch, nm, dev
+        self.layers = []
+        for s in specs:
+            i8 = s["dtype"] == "i8"
+            odt = od if od is not None else (nm.NM_OUT_I32 if i8 else nm.NM_OUT_F16)
+            if device_x:       # legs that are not compared with the oracle: activations drawn on the device
+                W = (inputs.w_i8 if i8 else inputs.w_f16)(s["O"], s["K"], s["n"], s["m"], s.get("name", ""), key, rank)
+                g = torch.Generator(device=dev).manual_seed(inputs.tensor_seed("x", s.get("name", ""), key, rank) & 0x7FFFFFFF)
+                Xd = (torch.randint(-128, 128, (s["T"], s["K"]), dtype=torch.int8, device=dev, generator=g) if i8 else
+                      (torch.randn((s["T"], s["K"]), dtype=torch.float32, device=dev, generator=g) * 0.02).half())
+                X = Xh = None
+            else:
+                X, W = inputs.make_layer(s, key, rank)
+                Xh = torch.from_numpy(X).pin_memory() if host_x else None
+                Xd = torch.from_numpy(X).to(dev)
+            w = nm.nm_compress(W, s["n"], s["m"])
+            plan = nm.nm_plan_create(s["T"], w, odt, dev.index)
+            Yd = torch.empty((s["T"], s["O"]), dtype=nm._out_torch_dtype(odt), device=dev)
+            ws = torch.empty(max(int(plan.workspace_bytes), 256), dtype=torch.uint8, device=dev)
+            self.layers.append(dict(spec=s, w=w, plan=plan, Xh=Xh, Xd=Xd, Yd=Yd, ws=ws, W=W, X=X, od=odt))
+        self.status = torch.zeros(len(self.layers), dtype=torch.int32, device=dev)
+
+    def kernel_of(self, L):
+        p, dt = L["plan"], ("int8" if L["spec"]["dtype"] == "i8" else "fp16")
+        kind = {self.nm.NM_PATH_UMMA_SP24: "sparse 2:4", self.nm.NM_PATH_UMMA_DENSE: "dense"}.get(p.path, f"path {p.path}")
+        return f"{'nm_umma_pair_kernel' if p.cta_group == 2 else 'nm_umma_kernel'}<{dt}, {kind}>"
+
+    def step(self, sptr, only=None):
+        nm = self.nm
+        for i, L in enumerate(self.layers):
+            if only is not None and self.kernel_of(L) != only:
+                continue
+            st = nm.nm_spmm_raw(L["Xd"].data_ptr(), L["spec"]["K"], L["spec"]["T"], L["w"], L["plan"], L["Yd"].data_ptr(),
+                                L["spec"]["O"], L["od"], L["ws"].data_ptr(), L["ws"].numel(),
+                                self.status.data_ptr() + 4 * i, sptr)
+            if st != nm.NM_OK:
+                raise RuntimeError(f"nm_spmm failed: {nm.lib().nm_status_string(st).decode()}")
+
+    def graph(self, stream, only=None, reps=1):
+        torch = self.torch
+        with torch.cuda.stream(stream):
+            self.step(stream.cuda_stream, only)
+            stream.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                for _ in range(reps):
+                    self.step(stream.cuda_stream, only)
+            g.replay()
+            stream.synchronize()
+        return g
+
+    def status_words(self):
+        return [int(v) & 0xFFFFFFFF for v in self.status.cpu().tolist()]
+
+
+def time_graph(torch, stream, g, replays):
+    """Mean milliseconds per replay, CUDA events on the launching stream."""
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        a0.record(stream)
+        for _ in range(replays):
+            g.replay()
+        a1.record(stream)
+        stream.synchronize()
+    return a0.elapsed_time(a1) / replays
+
+
+def graph_of(torch, stream, fn, reps=1):
+    with torch.cuda.stream(stream):
+        fn()
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(reps):
+                fn()
+        g.replay()
+        stream.synchronize()
+    return g
+
+
+def library_dense_peak(torch, stream, dtype):
+    """Dense library GEMM 8192^3 on this GPU, best of 10 (burst), in T(FL)OPS."""
+    n = 8192
+    if dtype == "i8":
+        a = torch.randint(-128, 128, (n, n), dtype=torch.int8, device="cuda")
+        b = torch.randint(-128, 128, (n, n), dtype=torch.int8, device="cuda")
+        fn = lambda: torch._int_mm(a, b.t())          # noqa: E731  comparator only; never on the product path
+    else:
+        a = torch.randn((n, n), dtype=torch.float16, device="cuda")
+        b = torch.randn((n, n), dtype=torch.float16, device="cuda")
+        fn = lambda: torch.matmul(a, b.t())           # noqa: E731
+    g = graph_of(torch, stream, fn)
+    best = min(time_graph(torch, stream, g, 1) for _ in range(10))
+    return 2.0 * n ** 3 / (best * 1e-3) / 1e12
+
+
 # ---------------------------------------------------------------------------------- GPU arm
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--ref-rows", type=int, default=1024, help="token rows per GEMM the reference arm runs per step")
-    ap.add_argument("--cpu-rows", type=int, default=12608, help="token rows per GEMM of the cpu_baseline sample")
-    ap.add_argument("--per-layer", action="store_true", help="also print a per-GEMM table to stderr")
+    ap.add_argument("--workload", default="cfg2", choices=sorted(WORKLOADS))
+    ap.add_argument("--ref-rows", type=int, default=0, help="token rows per GEMM the reference arm runs per step (0: workload default)")
+    ap.add_argument("--cpu-rows", type=int, default=0, help="token rows per GEMM of the cpu_baseline sample (0: workload default)")
+    ap.add_argument("--per-layer", action="store_true", help="also print the per-GEMM table to stderr")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compare", action="store_true", help="skip the per-GEMM table and the cuBLAS comparator")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the cfg1 / FP16 / ViT-L legs")
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a CUDA graph")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    wl = WORKLOADS[args.workload]
     if args.impl == "reference":
-        return run_reference(args)
+        return run_reference(args, wl)
 
     import torch
     from paper_2607_12505_b200 import binding as nm
@@ -206,28 +275,11 @@ def main():
     dev = torch.device("cuda", local)
 
     # ---- synthetic workload: every GEMM owns its X, Y and packed W (step footprint >> L2)
-    specs = layer_specs()
-    layers = []
-    for s in specs:
-        X, W = inputs.make_layer(s, "bench", rank)
-        w = nm.nm_compress(W, s["n"], s["m"])
-        plan = nm.nm_plan_create(s["T"], w, nm.NM_OUT_I32, local)
-        Xh = torch.from_numpy(X).pin_memory()
-        Xd = Xh.to(dev)
-        Yd = torch.empty((s["T"], s["O"]), dtype=torch.int32, device=dev)
-        ws = torch.empty(max(int(plan.workspace_bytes), 256), dtype=torch.uint8, device=dev)
-        layers.append(dict(spec=s, w=w, plan=plan, Xh=Xh, Xd=Xd, Yd=Yd, ws=ws, W=W, X=X))
+    specs = wl["specs"]()
+    stack = Stack(torch, nm, specs, dev, "bench", rank, host_x=not args.no_e2e)
+    layers = stack.layers
     stream = torch.cuda.Stream(device=dev)
     sptr = stream.cuda_stream
-
-    def step(only=None):
-        for L in layers:
-            if only is not None and L["plan"].cta_group != only:
-                continue
-            st = nm.nm_spmm_raw(L["Xd"].data_ptr(), L["spec"]["K"], L["spec"]["T"], L["w"], L["plan"],
-                                L["Yd"].data_ptr(), L["spec"]["O"], nm.NM_OUT_I32, L["ws"].data_ptr(), L["ws"].numel(), 0, sptr)
-            if st != nm.NM_OK:
-                raise RuntimeError(f"nm_spmm failed: {nm.lib().nm_status_string(st).decode()}")
 
     def barrier():
         torch.cuda.synchronize()
@@ -238,24 +290,20 @@ def main():
     graph = None
     with torch.cuda.stream(stream):
         for _ in range(args.warmup):
-            step()
+            stack.step(sptr)
         stream.synchronize()
-        launches_per_step_before = nm.launch_count()
-        step()
-        launches_per_step = nm.launch_count() - launches_per_step_before
+        before = nm.launch_count()
+        stack.step(sptr)
+        launches_per_step = nm.launch_count() - before
         stream.synchronize()
-        if not args.no_graph:
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                step()
-            graph.replay()
-            stream.synchronize()
+    if not args.no_graph:
+        graph = stack.graph(stream)
 
     def run_step():
         if graph is not None:
             graph.replay()
         else:
-            step()
+            stack.step(sptr)
 
     # ---- timed region: K steps, CUDA events on the launching stream, max over ranks
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -276,31 +324,38 @@ def main():
     step_useful_ops = sum(useful_ops(s) for s in specs)
     step_bytes = sum(algorithmic_bytes(s) for s in specs)
     tops = world * step_dense_ops / (ms_per_step * 1e-3) / 1e12
+    status_words = stack.status_words()          # every launch of the warm-up and of the timed region ORs into these
 
-    # ---- cuBLAS dense comparator and per-GEMM table (outside the timed region).  Timed the same
-    # way as the product path: one CUDA graph per measurement, replayed, CUDA events around it.
-    per_layer = []
-    cublas_ms_step = None
-    copy_same_bytes = None
+    peak, peak_src = measured_peaks()
+
+    # ---- roofline of the dominant kernel (the one that moves most of the step's algorithmic bytes), timed over its own
+    # launches of the step (same order, one replayed graph) when the step mixes kernels
+    groups = {}
+    for L in layers:
+        g = groups.setdefault(stack.kernel_of(L), {"launches": 0, "bytes": 0.0})
+        g["launches"] += 2 if L["plan"].split_k > 1 else 1      # a split-K call adds its merge kernel
+        g["bytes"] += algorithmic_bytes(L["spec"])
+    dom = max(groups, key=lambda k: groups[k]["bytes"])
+    dom_bytes, dom_launches = groups[dom]["bytes"], groups[dom]["launches"]
+    if len(groups) == 1:
+        dom_us, scope = ms_per_step * 1e3, "the timed region (every launch of the step is this kernel)"
+    else:
+        gd = stack.graph(stream, only=dom)
+        dom_us = time_graph(torch, stream, gd, max(10, min(args.steps, 100))) * 1e3
+        others = ", ".join(f"{v['launches']} x {k}" for k, v in groups.items() if k != dom)
+        scope = f"this kernel's {dom_launches} launches of the step replayed as their own graph (the step's other launches: {others})"
+    achieved = dom_bytes / (dom_us * 1e-6) / 1e9
+    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- cuBLAS dense comparator, per-GEMM table, tensor-roofline leg (outside the timed region; rank 0).  Timed the
+    # same way as the product path: one CUDA graph per measurement, replayed, CUDA events around it.
+    per_layer, cublas, copy_same_bytes, tensor_roof, extra = [], None, None, None, {}
 
     def graph_us(fn, reps):
-        with torch.cuda.stream(stream):
-            fn()
-            stream.synchronize()
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=stream):
-                for _ in range(reps):
-                    fn()
-            g.replay()
-            stream.synchronize()
-            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a0.record(stream)
-            g.replay()
-            a1.record(stream)
-            stream.synchronize()
-        return a0.elapsed_time(a1) * 1e3 / reps
+        return time_graph(torch, stream, graph_of(torch, stream, fn, reps), 3) * 1e3 / reps
 
     if rank == 0 and not args.no_compare:
+        int8_peak = library_dense_peak(torch, stream, "i8")
         try:
             Wds = [torch.from_numpy(L["W"]).to(dev) for L in layers]
             outs = [None] * len(layers)
@@ -308,31 +363,55 @@ def main():
             def cublas_step():
                 for i, (L, Wd) in enumerate(zip(layers, Wds)):
                     outs[i] = torch._int_mm(L["Xd"], Wd.t())      # comparator only; never on the product path
-            cublas_ms_step = graph_us(cublas_step, 20) / 1e3
+            cublas_ms = graph_us(cublas_step, 5) / 1e3
+            del outs
+            cublas = {"ms_per_step": cublas_ms, "launch": "cuda_graph_replay", "library": "torch._int_mm (cuBLASLt heuristic)",
+                      "speedup_vs_cublas_dense": cublas_ms / ms_per_step}
+            seen = {}
             for L, Wd in zip(layers, Wds):
                 s = L["spec"]
+                key = (s["K"], s["O"], s["n"], s["m"])
+                if key in seen:                  # time every distinct (shape, ratio) once
+                    continue
                 us = graph_us(lambda: nm.nm_spmm_raw(L["Xd"].data_ptr(), s["K"], s["T"], L["w"], L["plan"], L["Yd"].data_ptr(),
-                                                     s["O"], nm.NM_OUT_I32, L["ws"].data_ptr(), L["ws"].numel(), 0, sptr), 10)
+                                                     s["O"], L["od"], L["ws"].data_ptr(), L["ws"].numel(), 0, sptr), 10)
                 cb_us = graph_us(lambda: torch._int_mm(L["Xd"], Wd.t()), 10)
-                per_layer.append({"name": s["name"], "us_warm": round(us, 2), "cublas_dense_us_warm": round(cb_us, 2),
-                                  "dense_tops": round(dense_ops(s) / us / 1e6, 1), "gbs": round(algorithmic_bytes(s) / us / 1e3, 1),
-                                  "plan": {k: v for k, v in L["plan"].as_dict().items() if k in ("path", "tile_t", "split_k", "stages", "cta_group", "issuers")}})
-            del Wds, outs
+                sp = L["plan"].path == nm.NM_PATH_UMMA_SP24
+                t_hbm = algorithmic_bytes(s) / (peak * 1e9) * 1e6
+                t_mma = dense_ops(s) / (int8_peak * (2.0 if sp else 1.0) * 1e12) * 1e6
+                row = {"name": s["name"], "us_warm": round(us, 2), "cublas_dense_us_warm": round(cb_us, 2),
+                       "speedup": round(cb_us / us, 3), "dense_tops": round(dense_ops(s) / us / 1e6, 1),
+                       "gbs": round(algorithmic_bytes(s) / us / 1e3, 1), "bound": "tensor" if t_mma > t_hbm else "hbm",
+                       "roofline_us": round(max(t_hbm, t_mma), 2), "frac_of_roofline": round(max(t_hbm, t_mma) / us, 3),
+                       "kernel": stack.kernel_of(L),
+                       "plan": {k: v for k, v in L["plan"].as_dict().items() if k in ("path", "tile_t", "split_k", "stages", "cta_group", "issuers")}}
+                seen[key] = row
+                per_layer.append(row)
+            del Wds
+            # fc2 (K = 3072 -> O = 768) is the operator of the step closest to the tensor ridge
+            rows = [r for r in per_layer if ".fc2." in r["name"]]
+            tensor_roof = {
+                "int8_dense_peak_tops_measured": round(int8_peak, 1), "peak_how": "torch._int_mm 8192^3, best of 10 graph replays, same run",
+                "sparse_peak": "2 x the dense peak", "nominal_dense_tops": NOMINAL_DENSE_TOPS["i8"],
+                "gemms": [{"name": r["name"], "dense_tops": r["dense_tops"], "bound": r["bound"],
+                           "frac_of_measured_peak": round(r["dense_tops"] / (int8_peak * (2 if r["plan"]["path"] == nm.NM_PATH_UMMA_SP24 else 1)), 3),
+                           "frac_of_nominal_peak": round(r["dense_tops"] / (NOMINAL_DENSE_TOPS["i8"] * (2 if r["plan"]["path"] == nm.NM_PATH_UMMA_SP24 else 1)), 3)}
+                          for r in rows]}
         except Exception as exc:
             print(f"[bench] cuBLAS comparator unavailable: {exc}", file=sys.stderr)
-        # Context for the roofline fraction: plain device copies that move the same bytes per
-        # launch (read half, write half), one per GEMM, replayed the same way.  A launch of this
-        # size pays its own ramp and tail, so a copy does not reach the long-run peak either.
+        # Context for the roofline fraction: plain device copies that move the same bytes per launch (read half,
+        # write half), one per GEMM, replayed the same way.
         try:
-            srcs = [torch.empty(int(algorithmic_bytes(L["spec"]) // 2), dtype=torch.uint8, device=dev) for L in layers]
+            srcs = [torch.empty(int(algorithmic_bytes(L["spec"]) // 2), dtype=torch.uint8, device=dev) for L in layers[:8]]
             dsts = [torch.empty_like(b) for b in srcs]
 
             def copy_step():
                 for a, b in zip(srcs, dsts):
                     b.copy_(a)
-            copy_ms_step = graph_us(copy_step, 20) / 1e3
-            copy_same_bytes = {"ms_per_step": copy_ms_step, "gbs": step_bytes / (copy_ms_step * 1e-3) / 1e9,
-                               "what": "12 device-to-device copies per step, each moving the algorithmic bytes of one GEMM"}
+            copy_ms = graph_us(copy_step, 5) / 1e3
+            cbytes = sum(2 * b.numel() for b in srcs)
+            copy_same_bytes = {"gbs": cbytes / (copy_ms * 1e-3) / 1e9, "frac_of_peak": cbytes / (copy_ms * 1e-3) / 1e9 / peak,
+                               "what": "device-to-device copies moving the algorithmic bytes of the step's first 8 GEMMs, one copy per GEMM, same graph timing"}
             del srcs, dsts
         except Exception as exc:
             print(f"[bench] copy comparator unavailable: {exc}", file=sys.stderr)
@@ -343,14 +422,13 @@ def main():
     # ---- end to end through the public API with host buffers
     e2e = None
     if not args.no_e2e:
-        Yh = [torch.empty((L["spec"]["T"], L["spec"]["O"]), dtype=torch.int32).pin_memory() for L in layers]
+        Yh = [torch.empty((L["spec"]["T"], L["spec"]["O"]), dtype=torch.int32, pin_memory=True) for L in layers]
         Xdev = [torch.empty_like(L["Xd"]) for L in layers]
         h2d = sum(L["Xh"].numel() for L in layers)
         d2h = sum(y.numel() * 4 for y in Yh)
-
-        # Three streams, as a serving loop would use them: host->device copies, the GEMMs and
-        # device->host copies overlap (PCIe is full duplex and the copy engines are separate);
-        # events carry the true dependencies, including the reuse of each buffer by the next step.
+        # Three streams, as a serving loop would use them: host->device copies, the GEMMs and device->host copies
+        # overlap (PCIe is full duplex and the copy engines are separate); events carry the true dependencies,
+        # including the reuse of each buffer by the next step.
         s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
         ev_in = [torch.cuda.Event() for _ in layers]
         ev_mm = [torch.cuda.Event() for _ in layers]
@@ -367,7 +445,7 @@ def main():
                     stream.wait_event(ev_in[i])
                     if not first:
                         stream.wait_event(ev_out[i])       # the previous step's result has left Yd
-                    nm.nm_spmm(xd, L["w"], plan=L["plan"], out=L["Yd"], out_dtype=nm.NM_OUT_I32, workspace=L["ws"], stream=stream)
+                    nm.nm_spmm(xd, L["w"], plan=L["plan"], out=L["Yd"], out_dtype=L["od"], workspace=L["ws"], stream=stream)
                     ev_mm[i].record(stream)
                 with torch.cuda.stream(s_out):
                     s_out.wait_event(ev_mm[i])
@@ -376,7 +454,7 @@ def main():
 
         e2e_step(True)
         torch.cuda.synchronize()
-        e2e_steps = max(3, min(args.steps, 10))
+        e2e_steps = 3
         barrier()
         e0.record(stream)
         for _ in range(e2e_steps):
@@ -388,7 +466,8 @@ def main():
         barrier()
         ems = sharding.max_over_ranks(e0.elapsed_time(e1), dev)
         e2e = {"value": world * step_dense_ops / (ems / e2e_steps * 1e-3) / 1e12, "unit": UNIT,
-               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": ems / e2e_steps}
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "ms_per_step": ems / e2e_steps,
+               "steps": e2e_steps}
         del Yh, Xdev
 
     if rank != 0:
@@ -396,76 +475,131 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- CPU oracle on a bounded sample (rank 0, N=1 only)
-    cpu = None
+    # ---- CPU oracle on a bounded sample (rank 0, N=1 only); its rows also verify what the timed kernels wrote
+    cpu, verified = None, {"status_words_zero": all(v == 0 for v in status_words), "status_words": sorted(set(status_words))}
     if world == 1 and not args.no_cpu:
-        run, sample_dense_ops, cores, desc = oracle_sample(specs, args.cpu_rows)
+        run_step()                                # Y of every layer as the timed launches leave it
+        torch.cuda.synchronize()
+        run, sample_dense_ops, cores, desc, outs = oracle_sample(specs, args.cpu_rows or wl["cpu_rows"], keep_outputs=True)
         t0 = time.perf_counter()
         run()
         dt = time.perf_counter() - t0
         cpu = {"value": sample_dense_ops / dt / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
                "seconds": round(dt, 2)}
+        mism = 0
+        for L, y in zip(layers, outs):
+            mism += int((L["Yd"][:y.shape[0]].cpu().numpy() != y).sum())
+        verified.update({"oracle_rows_per_gemm": int(outs[0].shape[0]), "gemms": len(outs), "mismatches": mism})
+    verified["ok"] = bool(verified["status_words_zero"] and verified.get("mismatches", 0) == 0)
+    del stack, layers, graph
 
-    peak, peak_src = measured_peaks()
-    # ---- roofline of the dominant kernel.  The planner may run some GEMMs of the step on the
-    # CTA-pair kernel; the fraction is reported for the kernel that moves most bytes, timed over
-    # its own launches of the step (same order, one replayed graph) when the step mixes kernels.
-    kernel_names = {1: "nm_umma_kernel<int8, sparse 2:4>", 2: "nm_umma_pair_kernel<int8, sparse 2:4>"}
-    groups = {}
-    for L in layers:
-        g = groups.setdefault(int(L["plan"].cta_group), {"launches": 0, "bytes": 0.0})
-        g["launches"] += 2 if L["plan"].split_k > 1 else 1      # a split-K call adds its merge kernel
-        g["bytes"] += algorithmic_bytes(L["spec"])
-    dom = max(groups, key=lambda k: groups[k]["bytes"])
-    dom_bytes, dom_launches = groups[dom]["bytes"], groups[dom]["launches"]
-    if len(groups) == 1:
-        dom_us, scope = ms_per_step * 1e3, "the timed region (every launch of the step is this kernel)"
-    else:
-        with torch.cuda.stream(stream):
-            step(only=dom)
-            stream.synchronize()
-            gd = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gd, stream=stream):
-                step(only=dom)
-            gd.replay()
-            stream.synchronize()
-            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            reps_d = 200
-            d0.record(stream)
-            for _ in range(reps_d):
-                gd.replay()
-            d1.record(stream)
-            stream.synchronize()
-        dom_us = d0.elapsed_time(d1) * 1e3 / reps_d
-        scope = "this kernel's %d launches of the step replayed as their own graph (the other %d launches run %s)" % (
-            dom_launches, int(launches_per_step) - dom_launches, ", ".join(kernel_names[k] for k in groups if k != dom))
-    achieved = dom_bytes / (dom_us * 1e-6) / 1e9
-    step_gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    # ---- further legs (rank 0, N = 1): the other configurations the metric names, each as one replayed CUDA graph
+    if world == 1 and not args.no_extra:
+        torch.cuda.empty_cache()
+        try:
+            extra.update(extra_legs(torch, nm, dev, stream, peak, args.workload))
+        except Exception as exc:
+            print(f"[bench] extra legs failed: {exc!r}", file=sys.stderr)
+
     line = {
-        "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": wl["metric"], "value": tops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "int8", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "tokens": specs[0]["T"], "gemms_per_step": len(specs), "out_dtype": "int32",
+        "config": {"workload": wl["name"], "tokens": specs[0]["T"], "gemms_per_step": len(specs), "out_dtype": "int32",
+                   "ratios": sorted({f"{s['n']}:{s['m']}" for s in specs}),
                    "l2": "inputs larger than L2: every GEMM owns its X/Y/W buffers, step footprint %.0f MB" % (step_bytes / 1e6),
-                   "launch": "cuda_graph_replay" if graph is not None else "eager"},
+                   "launch": "cuda_graph_replay" if not args.no_graph else "eager"},
         "useful_tops": world * step_useful_ops / (ms_per_step * 1e-3) / 1e12,
         "gpu_launches": int(launches_per_step * args.steps),
         "clocks": clocks,
         "e2e": e2e,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_DRAM_TRAFFIC_BYTES_PER_LAUNCH, "kernel": kernel_names[dom], "peak_source": peak_src,
+                     "traffic": NCU_DRAM_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload), "kernel": dom, "peak_source": peak_src,
+                     "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                      "measured_over": scope, "launches": int(dom_launches), "algorithmic_bytes_per_launch": dom_bytes / max(1, dom_launches),
                      "avg_launch_us": dom_us / max(1, dom_launches),
-                     "whole_step": {"launches": int(launches_per_step), "algorithmic_bytes": step_bytes, "achieved": step_gbs, "frac": step_gbs / peak}},
+                     "kernels_of_step": {k: {"launches": v["launches"], "algorithmic_bytes": v["bytes"]} for k, v in groups.items()},
+                     "whole_step": {"launches": int(launches_per_step), "algorithmic_bytes": step_bytes, "achieved": step_gbs,
+                                    "frac": step_gbs / peak, "frac_of_nominal_8000": step_gbs / NOMINAL_HBM_GBS}},
         "cpu_baseline": cpu,
-        "cublas_dense": None if not cublas_ms_step else {"ms_per_step": cublas_ms_step, "launch": "cuda_graph_replay",
-                                                         "speedup_vs_cublas_dense": cublas_ms_step / ms_per_step},
+        "verified": verified,
+        "cublas_dense": cublas,
+        "tensor_roofline": tensor_roof,
         "copy_same_bytes": copy_same_bytes,
         "per_layer": per_layer,
     }
+    line.update(extra)
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def extra_legs(torch, nm, dev, stream, hbm_peak, main_workload):
+    """cfg1 step, cfg2 in FP16, the ViT-L batch-1 stack and one ViT-L batch-256 fc2 GEMM."""
+    out = {}
+
+    def run_stack(specs, key, reps):
+        st = Stack(torch, nm, specs, dev, key, device_x=True)
+        g = st.graph(stream)
+        ms = time_graph(torch, stream, g, reps)
+        words = st.status_words()
+        return st, ms, all(v == 0 for v in words)
+
+    # --- the DeiT-Small stack (12 GEMMs, 627 MB per step)
+    if main_workload != "cfg1":
+        specs = inputs.cfg1_layers()
+        st, ms, ok = run_stack(specs, "bench_cfg1", 50)
+        by = sum(algorithmic_bytes(s) for s in specs)
+        out["cfg1_step"] = {"workload": WORKLOADS["cfg1"]["name"], "ms_per_step": ms, "dense_tops": sum(dense_ops(s) for s in specs) / ms / 1e9,
+                            "gbs": by / ms / 1e6, "frac_of_hbm": by / ms / 1e6 / hbm_peak, "status_ok": ok}
+        del st
+        torch.cuda.empty_cache()
+
+    # --- the DeiT-Base stack in FP16 (fp32 accumulation, fp16 out), against torch.matmul on the same buffers
+    specs = inputs.cfg2_layers("f16")
+    st, ms, ok = run_stack(specs, "bench_f16", 10)
+    f16_peak = library_dense_peak(torch, stream, "f16")
+    Wds = [torch.from_numpy(L["W"]).to(dev) for L in st.layers]
+    outs = [None] * len(Wds)
+
+    def cublas_step():
+        for i, (L, Wd) in enumerate(zip(st.layers, Wds)):
+            outs[i] = torch.matmul(L["Xd"], Wd.t())           # comparator only
+    cb_ms = time_graph(torch, stream, graph_of(torch, stream, cublas_step), 5)
+    ops = sum(dense_ops(s) for s in specs)
+    sp_ops = sum(dense_ops(L["spec"]) for L in st.layers if L["plan"].path == nm.NM_PATH_UMMA_SP24)
+    out["cfg2_fp16"] = {"workload": "deit_base_12block_linear_stack_fp16_b128", "ms_per_step": ms, "dense_tflops": ops / ms / 1e9,
+                        "cublas_dense_ms_per_step": cb_ms, "speedup_vs_cublas_dense": cb_ms / ms,
+                        "fp16_dense_peak_tflops_measured": round(f16_peak, 1),
+                        "share_of_ops_on_sparse_mma": sp_ops / ops, "status_ok": ok}
+    del st, Wds, outs
+    torch.cuda.empty_cache()
+
+    # --- ViT-Large at batch 1: 24 blocks x {qkv, fc1, fc2} as 72 dependent launches with distinct weights (2:4, INT8)
+    specs = [dict(name=f"vit_l.b1.{blk}.{nme}", T=197, K=K, O=O, n=2, m=4, dtype="i8")
+             for blk in range(24) for (nme, K, O) in [("qkv", 1024, 3072), ("fc1", 1024, 4096), ("fc2", 4096, 1024)]]
+    st, ms, ok = run_stack(specs, "bench_b1", 50)
+    by = sum(algorithmic_bytes(s) for s in specs)
+    out["vit_l_b1_stack"] = {"layers": len(specs), "us_per_layer": ms * 1e3 / len(specs), "ms_per_pass": ms, "algorithmic_mb": by / 1e6,
+                             "gbs": by / ms / 1e6, "frac_of_hbm": by / ms / 1e6 / hbm_peak, "status_ok": ok,
+                             "what": "one CUDA graph of the 72 linear layers, every layer its own packed weight, X and Y"}
+    del st
+    torch.cuda.empty_cache()
+
+    # --- one large tensor-leaning GEMM: ViT-Large fc2 at batch 256 (T = 50432, K = 4096 -> O = 1024), 2:4 INT8
+    spec = dict(name="vit_l.b256.fc2.2:4.i8", T=50432, K=4096, O=1024, n=2, m=4, dtype="i8")
+    int8_peak = library_dense_peak(torch, stream, "i8")
+    st = Stack(torch, nm, [spec, dict(spec, name=spec["name"] + ".b")], dev, "bench_b256", device_x=True)     # two buffer sets: 830 MB > L2
+    ms = time_graph(torch, stream, st.graph(stream, reps=5), 3) / 10
+    L = st.layers[0]
+    Wd = torch.from_numpy(L["W"]).to(dev)
+    cb = time_graph(torch, stream, graph_of(torch, stream, lambda: torch._int_mm(L["Xd"], Wd.t()), 10), 3) / 10
+    t_ops = dense_ops(spec) / ms / 1e9
+    out["vit_l_b256_fc2"] = {"us": ms * 1e3, "dense_tops": t_ops, "cublas_dense_us": cb * 1e3, "speedup_vs_cublas_dense": cb / ms,
+                             "frac_of_sparse_peak_measured": t_ops / (2 * int8_peak), "frac_of_sparse_peak_nominal_9000": t_ops / 9000.0,
+                             "int8_dense_peak_tops_measured": round(int8_peak, 1), "gbs": algorithmic_bytes(spec) / ms / 1e6,
+                             "frac_of_hbm": algorithmic_bytes(spec) / ms / 1e6 / hbm_peak, "status_ok": all(v == 0 for v in st.status_words())}
+    return out
 
 
 if __name__ == "__main__":

@@ -1,6 +1,6 @@
 """Calibrate and validate the latency predictor of Section 5.1 on one B200.
 
-    python -m paper_2607_12505_b200.predictor_eval [--model deit_b] [--batch 64] [--fit 40] [--test 24]
+    python -m bench.predictor_eval [--model deit_b] [--batch 64] [--fit 40] [--test 24]
 
 1. Table: nm_latency_table over the model's operator shapes x the ratios N:8, N = 1..8
    (INT8 -> INT32), i.e. the (shape, sparsity) lookup table.
@@ -19,18 +19,7 @@ import json
 
 import numpy as np
 
-MODELS = {
-    # name: (blocks, hidden, tokens per image)
-    "deit_s": (12, 384, 197),
-    "deit_b": (12, 768, 197),
-    "vit_l": (24, 1024, 197),
-}
-
-
-def layer_shapes(model: str):
-    blocks, d, _ = MODELS[model]
-    per_block = [("qkv", d, 3 * d), ("proj", d, d), ("fc1", d, 4 * d), ("fc2", 4 * d, d)]
-    return [(f"b{b}.{name}", K, O) for b in range(blocks) for (name, K, O) in per_block]
+from paper_2607_12505_b200.inputs import MODELS, layer_shapes  # noqa: E402,F401
 
 
 class Stack:
@@ -39,8 +28,8 @@ class Stack:
 
     def __init__(self, model="deit_b", batch=64, reps=20, blocks=None):
         import torch
-        from . import binding as nm
-        from . import inputs
+        from paper_2607_12505_b200 import binding as nm
+        from paper_2607_12505_b200 import inputs
         self.torch, self.nm, self.inputs = torch, nm, inputs
         self.reps = reps
         self.T = batch * MODELS[model][2]
@@ -117,7 +106,7 @@ def evaluate(model="deit_b", batch=64, fit=40, test=24, group="layer", reps=20, 
     """Runs the three steps; returns (summary dict, design matrix [S, n_coef], measured [S])."""
     import argparse as _ap
     args = _ap.Namespace(model=model, batch=batch, fit=fit, test=test, group=group, reps=reps, seed=seed)
-    from . import binding as nm
+    from paper_2607_12505_b200 import binding as nm
     stack = Stack(model, batch, reps, blocks)
     T, L, layers, lut, shapes, measure = stack.T, stack.L, stack.layers, stack.lut, stack.shapes, stack.measure
 

@@ -1,6 +1,6 @@
 """Run one GEMM shape through nm_spmm repeatedly (for timing sweeps and ncu captures).
 
-    python -m paper_2607_12505_b200.profile_case --T 12608 --O 1152 --K 384 --nm 2:4 \
+    python -m bench.profile_case --T 12608 --O 1152 --K 384 --nm 2:4 \
         [--dtype i8|f16] [--out i32|f32|f16] [--reps 20] [--rotate 4] [--tile-t 128] \
         [--stages 2] [--split-k 1] [--path simt|dense|sp24]
 
@@ -41,8 +41,8 @@ def main():
     args = ap.parse_args()
 
     import torch
-    from . import binding as nm
-    from . import inputs
+    from paper_2607_12505_b200 import binding as nm
+    from paper_2607_12505_b200 import inputs
 
     n, m = (int(v) for v in args.nm.split(":"))
     spec = dict(T=args.T, O=args.O, K=args.K, n=n, m=m, dtype=args.dtype, name="profile")

@@ -1,6 +1,6 @@
 """Per-shape performance report over the benchmark configurations (one B200).
 
-    python -m paper_2607_12505_b200.report [--configs cfg1,cfg2,cfg4] [--reps 20] [--out report.json]
+    python -m bench.report [--configs cfg1,cfg2,cfg4] [--reps 20] [--out report.json]
 
 For every distinct (layer shape, n:m, dtype) of the selected configurations it times nm_spmm
 under the library's own plan and dense cuBLAS (torch._int_mm / torch.matmul) on the same
@@ -9,7 +9,9 @@ larger than L2 -- and prints microseconds, useful and dense-equivalent T(FL)OPS,
 algorithmic bytes, and the fraction of the HBM and tensor rooflines.  The tensor peaks are
 measured in the same run (dense library GEMM 8192^3; the sparse peak is taken as twice that).
 It also times the small-batch weight-streaming case as a stack: the 72 distinct linear layers
-of ViT-L at batch 1 in one graph, bytes over time.
+of ViT-L at batch 1 in one graph, bytes over time.  The SM clock and the throttle reasons seen
+while each configuration was timed are printed and stored with its rows (a group taken under a
+thermal or hardware slowdown is to be re-run).
 """
 from __future__ import annotations
 
@@ -74,10 +76,13 @@ def main():
     args = ap.parse_args()
 
     import torch
-    from . import binding as nm
-    from . import inputs
+    from paper_2607_12505_b200 import binding as nm
+    from paper_2607_12505_b200 import inputs
 
+    from bench.clocks import ClockSampler
     stream = torch.cuda.Stream()
+    sampler = ClockSampler(torch.cuda.current_device()).start()
+    clock_groups = {}
     hbm = 6450.9
     peaks_file = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
     if os.path.exists(peaks_file):
@@ -96,6 +101,7 @@ def main():
     for cname in ([] if args.stack_only else args.configs.split(",")):
         seen = set()
         count = 0
+        mark = sampler.mark()
         for s in cfgs[cname]:
             key = (s["T"], s["K"], s["O"], s["n"], s["m"], s["dtype"])
             if key in seen:
@@ -141,11 +147,15 @@ def main():
             rows.append(row)
             print(json.dumps(row))
             del Xs, Ys, Wd, w
+        # clocks and throttle reasons seen while this configuration's rows were timed (read-only query)
+        clock_groups[cname] = sampler.summary(since=mark)
+        print(json.dumps({"clocks": cname, **clock_groups[cname]}))
 
     # ---- the fused requantising epilogue (INT8 in, INT8 out) on the INT8 2:4 layers of cfg1 / cfg2:
     # one byte per output instead of four moves these GEMMs from the HBM towards the tensor roofline
     if not args.stack_only and not args.max_shapes:
         seen = set()
+        mark = sampler.mark()
         for cname in [c for c in args.configs.split(",") if c in ("cfg1", "cfg2")]:
             for s in cfgs[cname]:
                 key = (s["T"], s["K"], s["O"])
@@ -176,11 +186,14 @@ def main():
                 rows.append(row)
                 print(json.dumps(row))
                 del Xs, Ys, w
+        clock_groups["int8_out"] = sampler.summary(since=mark)
+        print(json.dumps({"clocks": "int8_out", **clock_groups["int8_out"]}))
 
     # ---- small-batch weight streaming measured over a stack of distinct layers (ViT-L, batch 1)
     stack = None
     if "cfg4" in args.configs or args.stack_only:
         T = 197
+        mark = sampler.mark()
         for (n, m) in [(2, 4), (1, 8)]:
             layers = []
             for blk in range(24):
@@ -207,8 +220,11 @@ def main():
             print(json.dumps(stack))
             rows.append(stack)
             del layers
+        clock_groups["vit_l_b1_stack"] = sampler.summary(since=mark)
+        print(json.dumps({"clocks": "vit_l_b1_stack", **clock_groups["vit_l_b1_stack"]}))
+    sampler.stop()
     if args.out:
-        json.dump(dict(hbm_gbs=hbm, peaks=peaks, rows=rows), open(args.out, "w"))
+        json.dump(dict(hbm_gbs=hbm, peaks=peaks, clocks=clock_groups, rows=rows), open(args.out, "w"))
 
 
 if __name__ == "__main__":

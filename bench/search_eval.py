@@ -1,7 +1,7 @@
 """Close the loop of Section 5 on one B200: table -> calibrated predictor -> Algorithm 1 ->
 measure what the search chose.
 
-    python -m paper_2607_12505_b200.search_eval [--model deit_b] [--batch 64] [--budgets 0.8,0.85,0.9,0.95]
+    python -m bench.search_eval [--model deit_b] [--batch 64] [--budgets 0.8,0.85,0.9,0.95]
 
 The fitness is synthetic (the paper's is the accuracy inherited from a trained supernet, which
 needs ImageNet and trained weights): separable, increasing and concave in the level of each
@@ -33,8 +33,8 @@ def main():
     ap.add_argument("--out", default=None)
     args = ap.parse_args()
 
-    from . import binding as nm
-    from .predictor_eval import Stack
+    from paper_2607_12505_b200 import binding as nm
+    from bench.predictor_eval import Stack
 
     stack = Stack(args.model, args.batch, args.reps)
     L = stack.L

@@ -1,6 +1,6 @@
 """Sustained throughput of tensor-bound GEMMs under the board power limit, with the clocks seen.
 
-    python -m paper_2607_12505_b200.sustained [--seconds 4] [--out sustained.json]
+    python -m bench.sustained [--seconds 4] [--out sustained.json]
 
 A graph of 20 back-to-back calls lasts a few milliseconds: short enough for the GPU to run it at
 its maximum clock.  A kernel that keeps the tensor cores busy for seconds is throttled to the
@@ -80,8 +80,8 @@ def main():
     args = ap.parse_args()
 
     import torch
-    from . import binding as nm
-    from . import inputs
+    from paper_2607_12505_b200 import binding as nm
+    from paper_2607_12505_b200 import inputs
 
     stream = torch.cuda.Stream()
     index = torch.cuda.current_device()

@@ -140,8 +140,18 @@ typedef struct nm_plan {
   int32_t issuers;          /* single-CTA tcgen05 paths: 1, or 2 = a second warp issues the odd K steps of every
                                tile into a second accumulator that the epilogue adds (0 is read as 1) */
   int32_t merge;            /* NM_MERGE_*: where the split_k partial sums of a tile meet (ignored when split_k == 1) */
-  int32_t reserved;         /* 0 */
+  int32_t reserved;         /* 0, or NM_PLAN_DIAG_* bits */
 } nm_plan;
+
+/* Diagnostic bit of nm_plan.reserved (single-CTA tcgen05 paths; ignored elsewhere).  Every wait in
+ * the kernels is a bounded poll: when one runs out, the CTA ORs (NM_ERR_TIMEOUT | site << 8) into
+ * the status word, raises a CTA-wide abort flag, lets the copies it issued land, frees its tensor
+ * memory and returns.  NM_PLAN_DIAG_STALL makes that path observable without a fault: CTA 0 arms
+ * the barrier of its first K step for 16 bytes more than it requests, so every copy lands, that one
+ * barrier never completes, and the issuing warp's wait (site 2) runs out after a poll budget cut to
+ * about a millisecond for this launch.  The call returns normally, the status word reads
+ * NM_ERR_TIMEOUT | 2 << 8, Y is unspecified, and the stream stays usable. */
+enum { NM_PLAN_DIAG_STALL = 1 };
 
 /* One row of the latency table (Section 5.1: per-operator sparsity-latency LUT). */
 typedef struct nm_latency_row {
@@ -280,10 +290,14 @@ NM_API nm_status nm_spmm_ex(const void* X_dev, int64_t ldx, int T, const nm_weig
  * fixed array of NM_STATIC_SCRATCH_BYTES that is part of the library image; every GPU
  * that loads the library holds that array until the process exits.
  *   - Arguments are those of nm_spmm without the workspace pair; X, Y and the packed
- *     weight are still the caller's buffers.  plan may be NULL (automatic plan).
- *   - A plan whose workspace_bytes exceeds NM_STATIC_SCRATCH_BYTES returns
+ *     weight are still the caller's buffers.
+ *   - An explicit plan whose workspace_bytes exceeds NM_STATIC_SCRATCH_BYTES returns
  *     NM_ERR_WORKSPACE; nothing is launched.  Plans with split_k == 1 need no scratch
  *     and always pass.
+ *   - plan may be NULL: the automatic plan is then made against the fixed array and
+ *     degrades like nm_spmm's (no split-K, or on-chip decode instead of the dense scratch
+ *     copy, when the array is too small; the CUDA-core path when X or Y is not 16-byte
+ *     aligned): it never fails on scratch size or alignment.
  *   - No cudaMalloc / cudaFree / allocating library routine is called, on any path.
  *   - The first call on each device looks up the array's device address (with that device
  *     current); make that first call outside any stream capture.

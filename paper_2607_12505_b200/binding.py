@@ -24,6 +24,7 @@ NM_IMG_CANONICAL, NM_IMG_HW24, NM_IMG_DENSE, NM_IMG_AUTO = 1, 2, 4, 0x80000000
 NM_PATH_SIMT, NM_PATH_UMMA_DENSE, NM_PATH_UMMA_SP24, NM_PATH_UMMA_DECODE, NM_PATH_UMMA_EXPAND = 0, 1, 2, 3, 4
 NM_RES_NONE, NM_RES_X, NM_RES_W = 0, 1, 2
 NM_MERGE_WORKSPACE, NM_MERGE_CLUSTER = 0, 1
+NM_PLAN_DIAG_STALL = 1
 
 EXPORTS = [
     "nm_packed_size", "nm_compress", "nm_compress_host", "nm_prune_magnitude", "nm_decompress",

@@ -71,7 +71,9 @@ nm_status launch_umma(const SpmmArgs& a);
 nm_status launch_umma_pair(const SpmmArgs& a, bool* handled);   // cta_group::2 variant; may decline
 void count_launch(int n = 1);
 
-// Bytes of split-K scratch a plan needs: partial tiles + one ticket counter per output tile.
+// Bytes of split-K scratch a plan needs: one raw 32-bit slice [t_pad x O] per K split (t_pad =
+// token rows rounded up to whole tiles).  The merge pass reads only rows t < T and columns o < O
+// of every slice, all of which the same call's GEMM kernel writes first: nothing has to be zeroed.
 uint64_t splitk_workspace_bytes(int T, int O, int tile_t, int split_k);
 
 }  // namespace nm

@@ -77,6 +77,8 @@ struct UmmaParams {
   int cluster_merge;        // split-K: the K slices of a tile are the CTAs of one cluster and meet on chip
   uint32_t recv_bytes;      // ... bytes of shared memory that receive the other slices' partials
   int t_pad;                // split-K: token rows per slice (tiles_t * tile_t)
+  uint32_t spin_limit;      // polls after which a bounded wait gives up
+  int diag_stall;           // diagnostic (NM_PLAN_DIAG_STALL): CTA 0 arms its first K step for 16 bytes that never come
   uint32_t* status;
   // decode path: the canonical image (values + bit-packed positions)
   const uint8_t* canon_vals; const uint8_t* canon_idx;
@@ -117,7 +119,6 @@ __host__ __device__ inline uint32_t cluster_recv_bytes(int tile_t, int split) {
 
 struct ItemCoord {
   int o0, t0, ks_begin, nsteps, z;
-  uint32_t tile;     // index into the split-K ticket array
   int key;           // identifies the resident operand this item needs
 };
 // Work items of one CTA: item(n) = first + n * stride, n < count.  Streaming mode strides over
@@ -144,7 +145,6 @@ __device__ __forceinline__ ItemCoord decode_item(const UmmaParams& p, int item) 
   int ot, tt;
   if (p.resident == NM_RES_W) { ot = tile / p.tiles_t; tt = tile % p.tiles_t; }   // token tiles fastest
   else { tt = tile / p.tiles_o; ot = tile % p.tiles_o; }                            // out-feature tiles fastest
-  c.tile = (uint32_t)(tt * p.tiles_o + ot);
   c.o0 = ot * kTileO;
   c.t0 = tt * p.tile_t;
   c.key = p.resident == NM_RES_W ? ot : tt;
@@ -177,7 +177,6 @@ struct ItemWalker {
     if (!fast) return decode_item(p, item);
     ItemCoord c;
     c.z = z;
-    c.tile = (uint32_t)(tt * p.tiles_o + ot);
     c.o0 = ot * kTileO;
     c.t0 = tt * p.tile_t;
     c.key = tt;
@@ -227,7 +226,13 @@ __device__ __forceinline__ void decode_row_kstep(const UmmaParams& p, uint32_t t
   const int g_valid = (row < p.O) ? max(0, min(p.G - g0, groups_per_step)) : 0;
 
   // ---- fetch: aligned 16-byte windows over the value bytes and the position bits of the step
-  uint32_t vbuf[36], ibuf[24];
+  // Window sizes: a K step is 128 bytes of the dense row, i.e. at most 128 kept values of one
+  // byte (n = m) or 64 of two, so at most 128 value bytes plus 15 bytes of window misalignment
+  // = 143 -> 9 loads of 16; its position bits are at most 128 * 4 / 8 = 64 bytes (m = 16, n = 15,
+  // one-byte values) plus 15 -> 79 -> 5 loads, 6 issued.  A field that ends in the last fetched
+  // word still forms `two` from the word after it, so the index buffer keeps one spare, zeroed word.
+  uint32_t vbuf[36], ibuf[25];
+  ibuf[24] = 0u;
   const size_t v_begin = (size_t)g0 * p.n * eb, v_end = v_begin + (size_t)g_valid * p.n * eb;
   const size_t i_begin = ((size_t)g0 * p.n * p.b) >> 3, i_end = (((size_t)(g0 + g_valid) * p.n * p.b) + 7) >> 3;
   const size_t v_win = v_begin & ~(size_t)15, i_win = i_begin & ~(size_t)15;
@@ -313,6 +318,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(
       gen_base + p.res_bytes + ring_bytes + kEpiWarps * kPatchBufs * kPatchBytes + p.recv_bytes + 16u * p.stages + 8u * (2u * kMaxAcc + 3u));
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  const WaitCtx wctx{abort_flag, p.status, p.spin_limit};
   // where the A part (W values, then metadata) and the B part (X) of K step ks / ring stage s live
   const uint32_t a_off_in_stage = p.resident == NM_RES_X ? 0u : b_part_bytes<DT, SP>(p.tile_t);
 
@@ -368,7 +374,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // grid-dependency wait: in a stack of small-batch layers the weight fetch of layer i+1
       // overlaps layer i.  X is only touched after the wait.
       int pre = 0;
-      if (p.resident == NM_RES_NONE && !DEC && !p.w_fresh && R.count > 0) {
+      if (p.resident == NM_RES_NONE && !DEC && !p.w_fresh && !p.diag_stall && R.count > 0) {
         const ItemCoord c0 = decode_item(p, R.first);
         const uint8_t* meta0 = SP ? p.meta + ((size_t)(c0.o0 / kTileO) * p.meta_kblocks) * kMetaBlockBytes : nullptr;
         pre = min(p.stages, c0.nsteps);
@@ -393,6 +399,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       pdl_wait_prior_grid();      // X (and the workspace) may be written by the previous kernel
       uint32_t rloads = 0, s = 0, ph = 0, st = ring_base;
+      uint32_t armed = 0;          // ring stages armed so far (K steps whose loads were issued)
       bool wrapped = false;
       int prev_key = -1;
       bool ok = true;
@@ -402,7 +409,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (p.resident != NM_RES_NONE && c.key != prev_key && !(DEC && p.resident == NM_RES_W)) {
           // (re)load the resident operand, all K steps, once the MMAs that read the old one retired
           if (rloads >= 1u) {
-            ok = mbar_wait(bar_rempty, (rloads - 1u) & 1u, abort_flag, p.status, 7);
+            ok = mbar_wait(bar_rempty, (rloads - 1u) & 1u, wctx, 7);
             if (!ok) break;
           }
           mbar_expect_tx(bar_rfull, p.res_bytes);
@@ -429,13 +436,17 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           // thread pays full latency for every integer division in its loop
           const bool w_prefetched = (n == 0 && i < pre);       // its W part is already in flight
           if (wrapped) {
-            ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag, p.status, 1);
+            ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, wctx, 1);
             if (!ok) break;
           }
           const uint32_t full = bar_full + 8u * s;
           const int ks = c.ks_begin + i;
+          // Diagnostic stall: the first K step of CTA 0 expects 16 bytes more than are sent.  Every
+          // copy that was issued lands; the barrier never completes, the issuing warp's bounded wait
+          // runs out and the CTA leaves through its abort path with nothing in flight.
+          const uint32_t extra = (p.diag_stall && blockIdx.x == 0 && n == 0 && i == 0) ? 16u : 0u;
           if (!w_prefetched)
-            mbar_expect_tx(full, (DEC && p.resident != NM_RES_W) ? sbytes - 16384u : sbytes);   // decoded A is not a TMA transfer
+            mbar_expect_tx(full, ((DEC && p.resident != NM_RES_W) ? sbytes - 16384u : sbytes) + extra);   // decoded A is not a TMA transfer
           if (p.resident != NM_RES_X) {            // B part streams
             if (SP) {
               tma_load_2d(st, &tmB, full, ks * 256, c.t0);
@@ -450,8 +461,23 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (SP) bulk_load(sa + 16384u, meta_src + (size_t)ks * meta_bytes_per_step<DT, SP>(),
                               meta_bytes_per_step<DT, SP>(), full);
           }
+          ++armed;
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; wrapped = true; st = ring_base; } else { st += sbytes; }
         }
+      }
+      // Before this thread leaves, every copy it issued must have landed: a CTA that takes the abort
+      // path gives up its shared memory while such a copy could still be writing to it.  Each stage's
+      // barrier completes when the bytes of its latest use have arrived (no later use can complete:
+      // this thread arms them), so a bounded wait on that phase of every armed stage is enough.  On
+      // the normal path the MMAs have consumed every stage and the waits return at once.
+      {
+        if (armed < (uint32_t)pre) armed = (uint32_t)pre;
+        const uint32_t ns = armed < (uint32_t)p.stages ? armed : (uint32_t)p.stages;
+        for (uint32_t d = 0; d < ns; ++d) {
+          const uint32_t last_use = (armed - 1u - d) / (uint32_t)p.stages;        // use count of stage (armed-1-d) % stages
+          mbar_wait_quiet(bar_full + 8u * ((armed - 1u - d) % (uint32_t)p.stages), last_use & 1u, p.spin_limit >> 2);
+        }
+        if (p.resident != NM_RES_NONE && rloads >= 1u) mbar_wait_quiet(bar_rfull, (rloads - 1u) & 1u, p.spin_limit >> 2);
       }
     }
   } else if (warp == 1 || (DUAL && warp == 2 + kEpiWarps)) {
@@ -461,8 +487,9 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // faster than ~45-60 cycles each, which bounds small tiles; two threads nearly double that, and
     // the fixed even/odd split keeps the summation order (and FP32 results) reproducible.
     const uint32_t which = warp == 1 ? 0u : 1u;
-    if (lane == 0) {
-      // ---------------- MMA issuer
+    {
+      // ---------------- MMA issuer: the whole warp walks the loop in lockstep; the tcgen05 wrappers
+      // elect the one lane that issues (see nm_umma_common.cuh), every lane polls the barriers.
       // instruction descriptor: D format (F32=1 / S32=2) at bit 4, A/B format at bits 7/10
       // (signed int8 = 1, f16 = 0), both operands K-major, N>>3 at bit 17, M>>4 at bit 24,
       // sparse flag at bit 2, metadata half selector (id2) at bits 0-1.
@@ -470,28 +497,34 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       idesc |= (DT == NM_I8) ? ((2u << 4) | (1u << 7) | (1u << 10)) : (1u << 4);
       if (SP) idesc |= 1u << 2;
       const ItemRange R = my_items(p);
-      // This thread alone paces the tensor core, and a lone thread pays the full latency of every
-      // dependent integer instruction: the ring position is advanced incrementally (no divisions),
-      // one descriptor per operand is built per K step and the four MMAs offset it by constants.
+      // This warp alone paces the tensor core: the ring position is advanced incrementally (no
+      // divisions), one descriptor per operand is built per K step and the four MMAs offset it by
+      // constants.
       uint32_t rloads = 0, s = 0, ph = 0, st = ring_base;
       const bool res_w = p.resident == NM_RES_W, res_x = p.resident == NM_RES_X;
       int prev_key = -1;
       bool ok = true;
       ItemWalker walk;
       walk.init(p, R);
+      // The producer is parked behind the previous grid of the stream until that grid has finished;
+      // waiting here too keeps that time out of this warp's bounded waits (it costs nothing once the
+      // producer is through).
+      pdl_wait_prior_grid();
       for (int n = 0; n < R.count && ok; ++n, walk.next(p)) {
         const uint32_t li = (uint32_t)n;
         const ItemCoord c = walk.get(p);
         const uint32_t buf = p.acc_bufs == 2 ? (li & 1u) : 0u, use = p.acc_bufs == 2 ? (li >> 1) : li;     // acc_bufs is 1 or 2
         if (p.resident != NM_RES_NONE && c.key != prev_key) {
-          ok = mbar_wait(bar_rfull, rloads & 1u, abort_flag, p.status, 8);
+          ok = mbar_wait(bar_rfull, rloads & 1u, wctx, 8);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
           ++rloads;
           prev_key = c.key;
         }
         if (use >= 1u) {     // the epilogue must have drained this accumulator buffer
-          ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, abort_flag, p.status, 4);
+          ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, wctx, 4);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
         }
@@ -505,7 +538,8 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; st = ring_base; } else { st += sbytes; }
             continue;
           }
-          ok = mbar_wait(bar_full + 8u * s, ph, abort_flag, p.status, 2);
+          ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2);
+          ok = __all_sync(0xffffffffu, ok);        // also re-converges the warp after the poll loop
           if (!ok) break;
           tc_fence_after();
           const int ks = c.ks_begin + i;
@@ -568,7 +602,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const ItemCoord c = decode_item(p, R.first + n * R.stride);
       const uint32_t buf = p.acc_bufs == 2 ? (li & 1u) : 0u, use = p.acc_bufs == 2 ? (li >> 1) : li;     // acc_bufs is 1 or 2
       uint32_t ok = 1;
-      if (lane == 0) ok = mbar_wait(bar_tfull + 8u * buf, use & 1u, abort_flag, p.status, 3) ? 1u : 0u;
+      if (lane == 0) ok = mbar_wait(bar_tfull + 8u * buf, use & 1u, wctx, 3) ? 1u : 0u;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       tc_fence_after();
@@ -609,7 +643,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                map_to_cta(bar_recv, owner));
             continue;
           }
-          const bool got = mbar_wait(bar_recv, 0u, abort_flag, p.status, 11);
+          const bool got = mbar_wait(bar_recv, 0u, wctx, 11);
           if (!__all_sync(0xffffffffu, got)) break;
           // own partial first, then the other ranks' in rank order: a fixed order for every unit
           for (uint32_t z = 0; z + 1u < split; ++z) {
@@ -698,13 +732,17 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint32_t g = 0, rfills = 0;
     int prev_key = -1;
     bool ok = true;
+    // The packed weight never depends on the previous grid, so decoding could start at once; but the
+    // stages these warps wait for are freed by MMAs that need X, which the producer only loads after
+    // the previous grid: waiting here keeps that grid's run time out of the bounded waits below.
+    pdl_wait_prior_grid();
     for (int n = 0; n < R.count && ok; ++n) {
       const ItemCoord c = decode_item(p, R.first + n * R.stride);
       if (p.resident == NM_RES_W) {
         if (c.key != prev_key) {
           // decode the whole W tile once for this run of token tiles
           if (rfills >= 1u) {
-            ok = mbar_wait(bar_rempty, (rfills - 1u) & 1u, abort_flag, p.status, 9);
+            ok = mbar_wait(bar_rempty, (rfills - 1u) & 1u, wctx, 9);
             if (!ok) break;
           }
           for (int ks = 0; ks < p.total_ksteps; ++ks)
@@ -720,7 +758,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int i = 0; i < c.nsteps; ++i, ++g) {
         const uint32_t s = g % (uint32_t)p.stages, nuse = g / (uint32_t)p.stages;
         if (nuse >= 1u) {
-          ok = mbar_wait(bar_empty + 8u * s, (nuse - 1u) & 1u, abort_flag, p.status, 10);
+          ok = mbar_wait(bar_empty + 8u * s, (nuse - 1u) & 1u, wctx, 10);
           if (!ok) break;
         }
         decode_row_kstep<DT>(p, ring_base + s * sbytes + a_off_in_stage, r, c.o0 + r, c.ks_begin + i, half);
@@ -955,6 +993,10 @@ nm_status launch_umma(const SpmmArgs& a) {
   p.epi_scale = a.epi.scale_dev; p.epi_bias = a.epi.bias_dev; p.epi_relu = a.epi.relu;
   if (p.out_i8 && !p.epi_scale) return NM_ERR_INVALID_ARG;
   p.status = a.status;
+  // diagnostic stall (see NM_PLAN_DIAG_STALL in nm.h): a short poll budget so that the stalled wait
+  // runs out in milliseconds
+  p.diag_stall = (pl.reserved & NM_PLAN_DIAG_STALL) ? 1 : 0;
+  p.spin_limit = p.diag_stall ? (1u << 14) : kSpinLimit;
   if (dec) {
     CanonGeom g;
     nm_status gs = canon_geom(w->O, w->K, w->n, w->m, w->dtype, &g);

@@ -41,6 +41,7 @@ struct PairParams {
   int out_i8;               // requantising epilogue (scale / bias / ReLU / saturate to int8)
   const float* epi_scale; const int32_t* epi_bias; int epi_relu;
   uint32_t tmem_cols;
+  uint32_t spin_limit;      // polls after which a bounded wait gives up
   uint32_t* status;
 };
 
@@ -59,21 +60,23 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
 }
 // commit of the pair's outstanding MMAs, arriving on the same-offset mbarrier of both CTAs
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+  asm volatile("{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+               "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
                ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
 __device__ __forceinline__ void tc_cp_128x128b_pair(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+  asm volatile("{\n\t.reg .pred e;\n\telect.sync _|e, 0xffffffff;\n\t"
+               "@e tcgen05.cp.cta_group::2.128x128b [%0], %1;\n\t}" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 template <int DT>
 __device__ __forceinline__ void tc_mma_dense_pair(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
   if (DT == NM_I8) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+    asm volatile("{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "@e tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
   } else {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+    asm volatile("{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "@e tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
   }
 }
@@ -81,12 +84,12 @@ template <int DT>
 __device__ __forceinline__ void tc_mma_sparse_pair(uint32_t d, uint64_t a, uint64_t b, uint32_t meta,
                                                    uint32_t idesc, uint32_t acc) {
   if (DT == NM_I8) {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                 "tcgen05.mma.sp.cta_group::2.kind::i8 [%0], %1, %2, [%3], %4, p;\n\t}"
+    asm volatile("{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "@e tcgen05.mma.sp.cta_group::2.kind::i8 [%0], %1, %2, [%3], %4, p;\n\t}"
                  ::"r"(d), "l"(a), "l"(b), "r"(meta), "r"(idesc), "r"(acc) : "memory");
   } else {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %5, 0;\n\t"
-                 "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
+    asm volatile("{\n\t.reg .pred p, e;\n\telect.sync _|e, 0xffffffff;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                 "@e tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n\t}"
                  ::"r"(d), "l"(a), "l"(b), "r"(meta), "r"(idesc), "r"(acc) : "memory");
   }
 }
@@ -122,6 +125,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(
       gen_base + ring_bytes + kEpiWarps2 * kPatchBytes2 + 16u * p.stages + 8u * 2u * kMaxAcc2);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  const WaitCtx wctx{abort_flag, p.status, p.spin_limit};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();            // 0 = leader (issues the MMAs), 1 = peer
@@ -186,7 +190,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       pdl_wait_prior_grid();
       bool ok = true, wrapped = false;
       // ring position kept incrementally (stage s, phase parity ph): no divisions in a lone thread
-      uint32_t s = 0, ph = 0, sa = smem_base;
+      uint32_t s = 0, ph = 0, sa = smem_base, armed = 0;
       for (int n = 0; n < my_count && ok; ++n) {
         const int item = pair + n * n_pairs;
         const int o0 = (item % p.tiles_o2) * 256 + (int)rank * 128;
@@ -197,7 +201,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (p.T - tile0 < p.tile_t) t0 = tile0 + (int)rank * (((p.T - tile0 + 31) & ~31) >> 1);
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
           if (wrapped) {
-            ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_flag, p.status, 1);
+            ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, wctx, 1);
             if (!ok) break;
           }
           const uint32_t full_leader = map_to_cta(bar_full + 8u * s, 0u);
@@ -216,13 +220,26 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int rows_per_step = (int)(meta_bytes2<DT, SP>() / 16u);
             tma_load_2d_pair(sm, &tmM, full_leader, 0, ((o0 / kTileO) * p.total_ksteps + ks) * rows_per_step);
           }
+          ++armed;
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; wrapped = true; sa = smem_base; } else { sa += sbytes; }
         }
       }
+      // Before the pair leaves, every copy its producers issued must have landed (a CTA on the abort
+      // path gives up its shared memory).  The full barriers live in the leader and count the bytes
+      // of both CTAs, so the leader waits (bounded) for the latest use of every armed stage; the peer
+      // cannot leave before the leader because of the cluster barrier at the end of the kernel.
+      if (rank == 0u) {
+        if (armed < (uint32_t)pre) armed = (uint32_t)pre;
+        const uint32_t ns = armed < (uint32_t)p.stages ? armed : (uint32_t)p.stages;
+        for (uint32_t d = 0; d < ns; ++d)
+          mbar_wait_quiet(bar_full + 8u * ((armed - 1u - d) % (uint32_t)p.stages),
+                          ((armed - 1u - d) / (uint32_t)p.stages) & 1u, p.spin_limit >> 2);
+      }
     }
   } else if (warp == 1) {
-    if (lane == 0 && rank == 0u) {
-      // ---------------- MMA issuer (leader only): M = 256 across the pair, N = tile_t
+    if (rank == 0u) {
+      // ---------------- MMA issuer (leader only): M = 256 across the pair, N = tile_t.  The whole
+      // warp walks the loop in lockstep; the tcgen05 wrappers elect the lane that issues.
       uint32_t idesc = ((uint32_t)(p.tile_t >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
       idesc |= (DT == NM_I8) ? ((2u << 4) | (1u << 7) | (1u << 10)) : (1u << 4);
       if (SP) idesc |= 1u << 2;
@@ -233,10 +250,12 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // token-tile index of this pair's items, advanced without a division per item
       const int step_t = n_pairs / p.tiles_o2, step_o = n_pairs % p.tiles_o2;
       int t_idx = pair / p.tiles_o2, o_idx = pair % p.tiles_o2;
+      pdl_wait_prior_grid();      // keeps the previous grid's run time out of the bounded waits below
       for (int n = 0; n < my_count && ok; ++n) {
         const uint32_t buf = (uint32_t)n % (uint32_t)p.acc_bufs, use = (uint32_t)n / (uint32_t)p.acc_bufs;
         if (use >= 1u) {       // both CTAs' epilogues must have drained this accumulator buffer
-          ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, abort_flag, p.status, 4);
+          ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, wctx, 4);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
         }
@@ -246,7 +265,8 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         t_idx += step_t; o_idx += step_o;
         if (o_idx >= p.tiles_o2) { o_idx -= p.tiles_o2; ++t_idx; }
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
-          ok = mbar_wait(bar_full + 8u * s, ph, abort_flag, p.status, 2);
+          ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2);
+          ok = __all_sync(0xffffffffu, ok);        // also re-converges the warp after the poll loop
           if (!ok) break;
           tc_fence_after();
           const uint32_t sm = sa + 16384u;
@@ -290,7 +310,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int t0 = (item / p.tiles_o2) * p.tile_t;
       const uint32_t buf = (uint32_t)n % (uint32_t)p.acc_bufs, use = (uint32_t)n / (uint32_t)p.acc_bufs;
       uint32_t ok = 1;
-      if (lane == 0) ok = mbar_wait(bar_tfull + 8u * buf, use & 1u, abort_flag, p.status, 3) ? 1u : 0u;
+      if (lane == 0) ok = mbar_wait(bar_tfull + 8u * buf, use & 1u, wctx, 3) ? 1u : 0u;
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       tc_fence_after();
@@ -455,6 +475,7 @@ nm_status launch_umma_pair(const SpmmArgs& a, bool* handled) {
   p.epi_scale = a.epi.scale_dev; p.epi_bias = a.epi.bias_dev; p.epi_relu = a.epi.relu;
   if (p.out_i8 && !p.epi_scale) return NM_ERR_INVALID_ARG;
   p.status = a.status;
+  p.spin_limit = kSpinLimit;
   p.w_fresh = a.w_fresh ? 1 : 0;
   p.tiles_o2 = ceil_div(w->O, 256);
   const int64_t items = (int64_t)p.tiles_o2 * ceil_div(a.T, pl.tile_t);

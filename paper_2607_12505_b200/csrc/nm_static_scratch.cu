@@ -46,17 +46,11 @@ extern "C" nm_status nm_spmm_static_scratch(const void* X_dev, int64_t ldx, int 
                                             const nm_plan* plan, void* Y_dev, int64_t ldy, nm_out_dtype od,
                                             uint32_t* status_dev, void* stream) {
   if (!w || w->magic != nm::kWeightMagic) return NM_ERR_INVALID_ARG;
-  nm_plan local;
-  if (!plan) {
-    int dev = 0, sms = nm::kDefaultSMs;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NM_ERR_CUDA;
-    nm_status st = nm_plan_shape(T, w->O, w->K, w->n, w->m, (nm_dtype)w->dtype, od, w->images, sms, &local);
-    if (st != NM_OK) return st;
-    plan = &local;
-  }
-  // the fixed array is all the scratch there is: a plan that needs more is refused, not shrunk
-  if (plan->workspace_bytes > (uint64_t)NM_STATIC_SCRATCH_BYTES) return NM_ERR_WORKSPACE;
+  // An explicit plan is taken at its word: if it needs more than the fixed array it is refused,
+  // not shrunk.  Without a plan nm_spmm plans against the size it is handed and degrades by itself
+  // (no split-K, on-chip decode instead of the dense scratch copy, the CUDA-core path for operands
+  // that TMA cannot address), exactly as it does for a caller-provided workspace.
+  if (plan && plan->workspace_bytes > (uint64_t)NM_STATIC_SCRATCH_BYTES) return NM_ERR_WORKSPACE;
   void* scratch = nullptr;
   nm_status st = scratch_address(&scratch);
   if (st != NM_OK) return st;

@@ -146,6 +146,20 @@ def cfg4_layers(dtypes=("i8", "f16"), batches=(1, 8, 64, 256)):
     return out
 
 
+MODELS = {
+    # name: (blocks, hidden, tokens per image)
+    "deit_s": (12, 384, 197),
+    "deit_b": (12, 768, 197),
+    "vit_l": (24, 1024, 197),
+}
+
+
+def layer_shapes(model: str):
+    """(name, K, O) of every linear layer of a ViT-family model, block by block."""
+    blocks, d, _ = MODELS[model]
+    return [(f"b{b}.{name}", K, O) for b in range(blocks) for (name, K, O) in vit_block_layers(d)]
+
+
 def make_layer(spec: dict, *key, at_most: bool = False):
     """(X, W) numpy arrays for one layer spec."""
     k = (spec.get("name", ""),) + key

@@ -12,7 +12,7 @@ import argparse
 import csv
 import json
 
-from .predictor_eval import MODELS, layer_shapes
+from .inputs import MODELS, layer_shapes
 
 FIELDS = ["T", "K", "O", "n", "m", "dtype", "out_dtype", "path", "tile_t", "split_k", "reps", "status", "us_mean", "us_min"]
 

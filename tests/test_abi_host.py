@@ -24,7 +24,10 @@ def test_library_exports_every_declared_symbol():
     for name in declared:
         assert hasattr(L, name), f"{name} not exported"
     assert L.nm_status_string(nm.NM_ERR_TIMEOUT) == b"NM_ERR_TIMEOUT"
-    assert nm.launch_count() == 0 or nm.launch_count() > 0
+    c0 = nm.launch_count()
+    assert isinstance(c0, int) and c0 >= 0
+    nm.nm_plan_shape(197, 384, 384, 2, 4, nm.NM_I8, nm.NM_OUT_I32, nm.NM_IMG_CANONICAL | nm.NM_IMG_HW24)
+    assert nm.launch_count() == c0, "host-only calls launch nothing"
 
 
 @pytest.mark.parametrize("n,m", NM_SET)
@@ -143,8 +146,17 @@ def test_plan_is_deterministic_and_follows_the_split_rule():
     # plenty of tiles -> no split; few tiles and a long K -> split grows (parallelism priority)
     small = nm.nm_plan_shape(197, 1024, 4096, 2, 4, nm.NM_I8, nm.NM_OUT_I32, imgs, 148)
     assert small.split_k > 1 and small.workspace_bytes > 0
-    tiles = -(-1024 // 128) * -(-197 // small.tile_t)
-    assert tiles * small.split_k >= 148 or small.split_k == 16 or True
+    # The split rule of Section 4.3 on this shape (16 K steps of 128 compressed bytes per row):
+    T, O, K, ksteps = 197, 1024, 4096, 16
+    tiles = -(-O // 128) * -(-T // small.tile_t)
+    in_bytes = T * K + O * (K // 2)
+    assert tiles < 148, "K is split only where one round of tiles leaves SMs idle"
+    assert ksteps // small.split_k >= 2, "controlled reduction: every slice keeps two K steps"
+    assert small.split_k * T * O * 4 <= 2 * in_bytes, "controlled reduction: partial sums do not dominate the traffic"
+    # parallelism priority: the split grows until the grid fills the SMs or the next candidate of the
+    # set {1, 2, 4, 8, 16} breaks one of the two conditions above
+    nxt = 2 * small.split_k
+    assert tiles * small.split_k >= 148 or nxt > 16 or ksteps // nxt < 2 or nxt * T * O * 4 > 2 * in_bytes
     # short K -> split stays 1 (controlled reduction)
     shortk = nm.nm_plan_shape(197, 384, 128, 2, 4, nm.NM_I8, nm.NM_OUT_I32, imgs, 148)
     assert shortk.split_k == 1

@@ -10,7 +10,7 @@ pytestmark = pytest.mark.gpu
 def test_calibration_on_a_small_stack():
     from oracle import nm_predictor_oracle as po
     from paper_2607_12505_b200 import binding as nm
-    from paper_2607_12505_b200 import predictor_eval
+    from bench import predictor_eval
 
     out, A, y = predictor_eval.evaluate(model="deit_s", batch=16, fit=14, test=6, group="operator", reps=10, seed=1, blocks=3)
     # the library's fit and the oracle's agree on the measured data
