@@ -144,13 +144,15 @@ typedef struct nm_plan {
 } nm_plan;
 
 /* Diagnostic bit of nm_plan.reserved (single-CTA tcgen05 paths; ignored elsewhere).  Every wait in
- * the kernels is a bounded poll: when one runs out, the CTA ORs (NM_ERR_TIMEOUT | site << 8) into
- * the status word, raises a CTA-wide abort flag, lets the copies it issued land, frees its tensor
- * memory and returns.  NM_PLAN_DIAG_STALL makes that path observable without a fault: CTA 0 arms
- * the barrier of its first K step for 16 bytes more than it requests, so every copy lands, that one
- * barrier never completes, and the issuing warp's wait (site 2) runs out after a poll budget cut to
- * about a millisecond for this launch.  The call returns normally, the status word reads
- * NM_ERR_TIMEOUT | 2 << 8, Y is unspecified, and the stream stays usable. */
+ * the kernels is a bounded poll: when one runs out, the CTA ORs (NM_ERR_TIMEOUT | 1 << (8 + site))
+ * into the status word, raises a CTA-wide abort flag, lets the copies it issued land, frees its
+ * tensor memory and returns.  NM_PLAN_DIAG_STALL makes that path observable without a fault: CTA 0
+ * arms the barrier of its first K step for 16 bytes more than it requests, so every copy lands,
+ * that one barrier never completes, and the waits behind it -- the issuing warp's for the stage
+ * (site 2), the epilogue's for the accumulator (site 3), the producer's for the stage to come free
+ * again (site 1) -- run out after a poll budget cut to milliseconds for this launch.  The call
+ * returns normally, the status word holds NM_ERR_TIMEOUT and the bit of whichever of those sites
+ * expired first, Y is unspecified, and the stream stays usable. */
 enum { NM_PLAN_DIAG_STALL = 1 };
 
 /* One row of the latency table (Section 5.1: per-operator sparsity-latency LUT). */
@@ -244,8 +246,11 @@ NM_API nm_status nm_plan_shape(int T, int O, int K, int n, int m, nm_dtype dt, n
  *   workspace_dev / workspace_bytes  device scratch >= plan->workspace_bytes
  *           (may be NULL/0 when the plan needs none); contents are overwritten
  *   status_dev  device, nullable: one uint32 the kernel ORs with
- *           (NM_ERR_TIMEOUT | site << 8) if a bounded wait expires; the caller
- *           zeroes it and reads it after synchronising.  Y is then unspecified.
+ *           (NM_ERR_TIMEOUT | 1 << (8 + site)) if a bounded wait expires (low byte: the status;
+ *           bits 9..19: which waits ran out -- 1 producer for a free ring stage, 2 issuing warp
+ *           for a loaded stage, 3 epilogue for an accumulator, 4 issuing warp for a drained
+ *           accumulator, 7-9 resident operand, 10 decode warps, 11 on-chip split-K merge); the
+ *           caller zeroes it and reads it after synchronising.  Y is then unspecified.
  * Enqueues on `stream` and returns; no synchronisation, no allocation.
  * The kernels are launched with programmatic stream serialisation: their prologue, and the
  * fetch of the first weight tiles, may overlap the tail of the previous kernel on the stream;

@@ -106,9 +106,12 @@ def lib() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB
-    if _build.is_stale():
-        path = _build.build()
+    if os.environ.get("NM_B200_TRACE") == "1":      # the trace build (phase stamps), for bench.trace_phases only
+        path = _build.build(trace=True)
+    else:
+        path = _build.LIB
+        if _build.is_stale():
+            path = _build.build()
     L = ctypes.CDLL(path)
     vp, i64, i32, u32, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_uint32, ctypes.c_size_t
     PW, PP = ctypes.POINTER(NMWeight), ctypes.POINTER(NMPlan)

@@ -12,6 +12,9 @@ namespace nm {
 static std::atomic<uint64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+static std::atomic<unsigned long long*> g_trace{nullptr};
+unsigned long long* trace_buffer() { return g_trace.load(std::memory_order_relaxed); }
+
 static uint32_t resolve_auto_images(int n, int m, bool clean24, int K, int eb) {
   uint32_t img = NM_IMG_CANONICAL;
   if (n == m) return img;                 // dense rows are already in the canonical values
@@ -64,6 +67,14 @@ const char* nm_status_string(nm_status s) {
 }
 
 uint64_t nm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+#ifdef NM_TRACE
+// Trace builds only (not declared in nm.h): device buffer of 16 x uint64 per CTA that the following
+// launches of the tcgen05 kernels stamp their phases into; nullptr switches the stamps off.
+__attribute__((visibility("default"))) void nm_trace_set_buffer(void* dev_buf) {
+  g_trace.store(static_cast<unsigned long long*>(dev_buf), std::memory_order_relaxed);
+}
+#endif
 
 size_t nm_packed_size(int O, int K, int n, int m, nm_dtype dt, uint32_t images) {
   PackLayout L;

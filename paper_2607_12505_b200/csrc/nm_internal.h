@@ -70,6 +70,8 @@ nm_status launch_simt(const SpmmArgs& a);
 nm_status launch_umma(const SpmmArgs& a);
 nm_status launch_umma_pair(const SpmmArgs& a, bool* handled);   // cta_group::2 variant; may decline
 void count_launch(int n = 1);
+// trace builds (-DNM_TRACE) only: the buffer the next launches stamp their phases into (nullptr: none)
+unsigned long long* trace_buffer();
 
 // Bytes of split-K scratch a plan needs: one raw 32-bit slice [t_pad x O] per K split (t_pad =
 // token rows rounded up to whole tiles).  The merge pass reads only rows t < T and columns o < O

@@ -79,6 +79,7 @@ struct UmmaParams {
   int t_pad;                // split-K: token rows per slice (tiles_t * tile_t)
   uint32_t spin_limit;      // polls after which a bounded wait gives up
   int diag_stall;           // diagnostic (NM_PLAN_DIAG_STALL): CTA 0 arms its first K step for 16 bytes that never come
+  unsigned long long* trace;   // phase stamps (trace builds only; nullptr otherwise)
   uint32_t* status;
   // decode path: the canonical image (values + bit-packed positions)
   const uint8_t* canon_vals; const uint8_t* canon_idx;
@@ -325,6 +326,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
+    NM_STAMP(p.trace, 0);
     pdl_launch_dependents();
     prefetch_tensormap(&tmA);
     prefetch_tensormap(&tmB);
@@ -362,6 +364,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   if (CLU) cluster_sync_all();     // every CTA's receive barrier is armed before anyone sends
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) NM_STAMP(p.trace, 1);
   const uint32_t acc_cols = (DUAL ? 2u : 1u) * (uint32_t)p.tile_t;          // columns of one accumulator buffer
   const uint32_t tmem_meta = tmem_base + (uint32_t)p.acc_bufs * acc_cols;    // metadata columns follow the accumulators
 
@@ -398,8 +401,11 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
       pdl_wait_prior_grid();      // X (and the workspace) may be written by the previous kernel
+      NM_STAMP(p.trace, 2);
+      NM_STAMP_VAL(p.trace, 12, R.count);
       uint32_t rloads = 0, s = 0, ph = 0, st = ring_base;
       uint32_t armed = 0;          // ring stages armed so far (K steps whose loads were issued)
+      long long cyc_empty = 0;     // trace builds: cycles spent waiting for a free stage
       bool wrapped = false;
       int prev_key = -1;
       bool ok = true;
@@ -436,7 +442,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           // thread pays full latency for every integer division in its loop
           const bool w_prefetched = (n == 0 && i < pre);       // its W part is already in flight
           if (wrapped) {
-            ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, wctx, 1);
+            NM_WAIT_TIMED(cyc_empty, ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, wctx, 1));
             if (!ok) break;
           }
           const uint32_t full = bar_full + 8u * s;
@@ -465,6 +471,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; wrapped = true; st = ring_base; } else { st += sbytes; }
         }
       }
+      NM_STAMP_VAL(p.trace, 15, cyc_empty);
       // Before this thread leaves, every copy it issued must have landed: a CTA that takes the abort
       // path gives up its shared memory while such a copy could still be writing to it.  Each stage's
       // barrier completes when the bytes of its latest use have arrived (no later use can complete:
@@ -506,6 +513,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       ItemWalker walk;
       walk.init(p, R);
+      long long cyc_full = 0, cyc_tempty = 0;      // trace builds: cycles spent inside the two waits of this warp
       // The producer is parked behind the previous grid of the stream until that grid has finished;
       // waiting here too keeps that time out of this warp's bounded waits (it costs nothing once the
       // producer is through).
@@ -523,7 +531,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           prev_key = c.key;
         }
         if (use >= 1u) {     // the epilogue must have drained this accumulator buffer
-          ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, wctx, 4);
+          NM_WAIT_TIMED(cyc_tempty, ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, wctx, 4));
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -538,10 +546,11 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; st = ring_base; } else { st += sbytes; }
             continue;
           }
-          ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2);
+          NM_WAIT_TIMED(cyc_full, ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2));
           ok = __all_sync(0xffffffffu, ok);        // also re-converges the warp after the poll loop
           if (!ok) break;
           tc_fence_after();
+          if (n == 0 && i == (int)which && lane == 0 && which == 0u) NM_STAMP(p.trace, 3);
           const int ks = c.ks_begin + i;
           const uint32_t slot = smem_base + (uint32_t)ks * slot_bytes;
           const uint32_t sa = res_w ? slot : st + a_off_in_stage;
@@ -578,12 +587,14 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         if (!ok) break;
         tc_commit(bar_tfull + 8u * buf);
+        if (lane == 0 && which == 0u) { if (n == 0) NM_STAMP(p.trace, 4); if (n + 1 == R.count) NM_STAMP(p.trace, 5); }
         if (p.resident != NM_RES_NONE) {
           // last tile on this resident operand: let the producer overwrite it once the MMAs retire
           const bool last_on_key = (n + 1 >= R.count) || decode_item(p, R.first + (n + 1) * R.stride).key != c.key;
           if (last_on_key) tc_commit(bar_rempty);
         }
       }
+      if (lane == 0 && which == 0u) { NM_STAMP_VAL(p.trace, 13, cyc_full); NM_STAMP_VAL(p.trace, 14, cyc_tempty); }
     }
   } else if (warp < 2 + kEpiWarps) {
     // ---------------- epilogue warps: quadrant q = TMEM lanes 32q..32q+31 (fixed by warp id),
@@ -596,16 +607,18 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int ob = (DT == NM_F16 && p.out_f16 && !ws_split) ? 2 : ((DT == NM_I8 && p.out_i8 && !ws_split) ? 1 : 4);
     const uint32_t crank = CLU ? cluster_cta_rank() : 0u;
     const ItemRange R = my_items(p);
+    long long cyc_tfull = 0;      // trace builds: cycles spent waiting for an accumulator
     pdl_wait_prior_grid();        // Y / workspace may still be in use by the previous kernel
     for (int n = 0; n < R.count; ++n) {
       const uint32_t li = (uint32_t)n;
       const ItemCoord c = decode_item(p, R.first + n * R.stride);
       const uint32_t buf = p.acc_bufs == 2 ? (li & 1u) : 0u, use = p.acc_bufs == 2 ? (li >> 1) : li;     // acc_bufs is 1 or 2
       uint32_t ok = 1;
-      if (lane == 0) ok = mbar_wait(bar_tfull + 8u * buf, use & 1u, wctx, 3) ? 1u : 0u;
+      if (lane == 0) NM_WAIT_TIMED(cyc_tfull, ok = mbar_wait(bar_tfull + 8u * buf, use & 1u, wctx, 3) ? 1u : 0u);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       tc_fence_after();
+      if (n == 0 && e == 0 && lane == 0) NM_STAMP(p.trace, 6);
       const int o_base = c.o0 + q * 32;
       const int o = o_base + lane;
       float q_scale = 1.0f;
@@ -719,11 +732,13 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8u * buf);
+      if (e == 0 && lane == 0) { if (n == 0) NM_STAMP(p.trace, 7); if (n + 1 == R.count) NM_STAMP(p.trace, 8); }
 
     }
     // the staging patches must outlive the stores' reads of them; the writes themselves complete
     // with the grid, which is what a dependent launch waits for
     if (p.epi_mode == kEpiTma && lane == 0) tma_store_wait_read();
+    if (e == 0 && lane == 0) { NM_STAMP(p.trace, 9); NM_STAMP_VAL(p.trace, 11, cyc_tfull); }
   } else if (DEC) {
     // ---------------- decode warps: thread r of 128 owns out-feature row o0 + r of the tile
     const int dt_id = (warp - (2 + kEpiWarps)) * 32 + lane;      // 0..255
@@ -774,6 +789,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // no CTA of a cluster leaves while a peer may still write into its shared memory or while its
   // own patches are being read by a copy towards a peer
   if (CLU) cluster_sync_all();
+  if (threadIdx.x == 0) NM_STAMP(p.trace, 10);
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
   }
@@ -897,6 +913,9 @@ nm_status launch_one(const SpmmArgs& a, const CUtensorMap& tmA, const CUtensorMa
   if (p.issuers == 2 && (DEC || p.resident != NM_RES_NONE || p.stages < 2 || 2u * (uint32_t)p.tile_t + meta_cols > 512u)) p.issuers = 1;
   p.acc_bufs = (int)((512u - meta_cols) / (uint32_t)(p.issuers * p.tile_t));
   if (p.acc_bufs > (int)kMaxAcc) p.acc_bufs = (int)kMaxAcc;
+  // a CTA that runs a single work item never rotates: one buffer, and half the tensor memory stays
+  // free for a CTA of the next launch that shares the SM under programmatic dependent launch
+  if (ceil_div(p.n_items, grid) <= 1) p.acc_bufs = 1;
   // An issuer waits on a ring stage by phase parity, which is only unambiguous while it cannot be
   // two uses of that stage ahead of the producer.  The issuer of the odd K steps observes no
   // barrier of the steps it skips; what bounds its lead is the accumulator hand-off (it can be
@@ -997,6 +1016,7 @@ nm_status launch_umma(const SpmmArgs& a) {
   // runs out in milliseconds
   p.diag_stall = (pl.reserved & NM_PLAN_DIAG_STALL) ? 1 : 0;
   p.spin_limit = p.diag_stall ? (1u << 14) : kSpinLimit;
+  p.trace = trace_buffer();
   if (dec) {
     CanonGeom g;
     nm_status gs = canon_geom(w->O, w->K, w->n, w->m, w->dtype, &g);

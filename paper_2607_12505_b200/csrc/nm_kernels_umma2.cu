@@ -42,6 +42,7 @@ struct PairParams {
   const float* epi_scale; const int32_t* epi_bias; int epi_relu;
   uint32_t tmem_cols;
   uint32_t spin_limit;      // polls after which a bounded wait gives up
+  unsigned long long* trace;   // phase stamps (trace builds only; nullptr otherwise)
   uint32_t* status;
 };
 
@@ -132,6 +133,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
+    NM_STAMP(p.trace, 0);
     pdl_launch_dependents();
     prefetch_tensormap(&tmA);
     prefetch_tensormap(&tmB);
@@ -157,6 +159,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   cluster_sync_all();                                  // barriers of both CTAs exist before any remote signal
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (threadIdx.x == 0) NM_STAMP(p.trace, 1);
   const uint32_t tmem_meta = tmem_base + (uint32_t)(p.acc_bufs * p.tile_t);
   const int my_count = (p.n_items > pair) ? (p.n_items - 1 - pair) / n_pairs + 1 : 0;
 
@@ -173,7 +176,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (rank == 0u) mbar_expect_tx(bar_full + 8u * (uint32_t)i, 2u * sbytes);
         tma_load_2d_pair(sa, &tmA, full_leader, i * 128, o0p);
         if (SP) tma_load_2d_pair(sa + 16384u, &tmM, full_leader, 0,
-                                 ((o0p / kTileO) * p.total_ksteps + i) * (int)(meta_bytes2<DT, SP>() / 16u));
+                                 ((o0p / kTileO) * p.total_ksteps + i) * (int)(meta_bytes2<DT, SP>() / 2048u));
       }
       // the X boxes of those K steps are pulled towards L2 (a hint, no data is consumed), so that
       // the first real loads after the wait do not pay the HBM latency
@@ -188,9 +191,12 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
       pdl_wait_prior_grid();
+      NM_STAMP(p.trace, 2);
+      NM_STAMP_VAL(p.trace, 12, my_count);
       bool ok = true, wrapped = false;
       // ring position kept incrementally (stage s, phase parity ph): no divisions in a lone thread
       uint32_t s = 0, ph = 0, sa = smem_base, armed = 0;
+      long long cyc_empty = 0;     // trace builds: cycles spent waiting for a free stage
       for (int n = 0; n < my_count && ok; ++n) {
         const int item = pair + n * n_pairs;
         const int o0 = (item % p.tiles_o2) * 256 + (int)rank * 128;
@@ -201,7 +207,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (p.T - tile0 < p.tile_t) t0 = tile0 + (int)rank * (((p.T - tile0 + 31) & ~31) >> 1);
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
           if (wrapped) {
-            ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, wctx, 1);
+            NM_WAIT_TIMED(cyc_empty, ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, wctx, 1));
             if (!ok) break;
           }
           const uint32_t full_leader = map_to_cta(bar_full + 8u * s, 0u);
@@ -217,13 +223,14 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             tma_load_2d_pair(sb, &tmB, full_leader, ks * 128, t0);
           }
           if (SP && !w_prefetched) {
-            const int rows_per_step = (int)(meta_bytes2<DT, SP>() / 16u);
-            tma_load_2d_pair(sm, &tmM, full_leader, 0, ((o0 / kTileO) * p.total_ksteps + ks) * rows_per_step);
+            const int blocks_per_step = (int)(meta_bytes2<DT, SP>() / 2048u);      // metadata map: one row per 2 KB block
+            tma_load_2d_pair(sm, &tmM, full_leader, 0, ((o0 / kTileO) * p.total_ksteps + ks) * blocks_per_step);
           }
           ++armed;
           if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; wrapped = true; sa = smem_base; } else { sa += sbytes; }
         }
       }
+      NM_STAMP_VAL(p.trace, 15, cyc_empty);
       // Before the pair leaves, every copy its producers issued must have landed (a CTA on the abort
       // path gives up its shared memory).  The full barriers live in the leader and count the bytes
       // of both CTAs, so the leader waits (bounded) for the latest use of every armed stage; the peer
@@ -250,11 +257,12 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // token-tile index of this pair's items, advanced without a division per item
       const int step_t = n_pairs / p.tiles_o2, step_o = n_pairs % p.tiles_o2;
       int t_idx = pair / p.tiles_o2, o_idx = pair % p.tiles_o2;
+      long long cyc_full = 0, cyc_tempty = 0;      // trace builds: cycles spent inside the two waits of this warp
       pdl_wait_prior_grid();      // keeps the previous grid's run time out of the bounded waits below
       for (int n = 0; n < my_count && ok; ++n) {
         const uint32_t buf = (uint32_t)n % (uint32_t)p.acc_bufs, use = (uint32_t)n / (uint32_t)p.acc_bufs;
         if (use >= 1u) {       // both CTAs' epilogues must have drained this accumulator buffer
-          ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, wctx, 4);
+          NM_WAIT_TIMED(cyc_tempty, ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, wctx, 4));
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -265,10 +273,11 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         t_idx += step_t; o_idx += step_o;
         if (o_idx >= p.tiles_o2) { o_idx -= p.tiles_o2; ++t_idx; }
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
-          ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2);
+          NM_WAIT_TIMED(cyc_full, ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2));
           ok = __all_sync(0xffffffffu, ok);        // also re-converges the warp after the poll loop
           if (!ok) break;
           tc_fence_after();
+          if (n == 0 && ks == 0 && lane == 0) NM_STAMP(p.trace, 3);
           const uint32_t sm = sa + 16384u;
           const uint32_t sb = sm + meta_bytes2<DT, SP>();
           const uint32_t meta_cols = tmem_meta + s * 8u;
@@ -296,13 +305,16 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         if (!ok) break;
         tc_commit_pair(bar_tfull + 8u * buf);          // accumulator ready in both CTAs
+        if (lane == 0) { if (n == 0) NM_STAMP(p.trace, 4); if (n + 1 == my_count) NM_STAMP(p.trace, 5); }
       }
+      if (lane == 0) { NM_STAMP_VAL(p.trace, 13, cyc_full); NM_STAMP_VAL(p.trace, 14, cyc_tempty); }
     }
   } else {
     // ---------------- epilogue warps (both CTAs): own 128 out-feature rows, all tile_t tokens
     const int e = warp - 2, q = warp & 3, h = e >> 2;
     const uint32_t patch = patches + (uint32_t)e * kPatchBytes2;
     const int ob = (DT == NM_F16 && p.out_f16) ? 2 : ((DT == NM_I8 && p.out_i8) ? 1 : 4);
+    long long cyc_tfull = 0;      // trace builds: cycles spent waiting for an accumulator
     pdl_wait_prior_grid();
     for (int n = 0; n < my_count; ++n) {
       const int item = pair + n * n_pairs;
@@ -310,10 +322,11 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int t0 = (item / p.tiles_o2) * p.tile_t;
       const uint32_t buf = (uint32_t)n % (uint32_t)p.acc_bufs, use = (uint32_t)n / (uint32_t)p.acc_bufs;
       uint32_t ok = 1;
-      if (lane == 0) ok = mbar_wait(bar_tfull + 8u * buf, use & 1u, wctx, 3) ? 1u : 0u;
+      if (lane == 0) NM_WAIT_TIMED(cyc_tfull, ok = mbar_wait(bar_tfull + 8u * buf, use & 1u, wctx, 3) ? 1u : 0u);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       tc_fence_after();
+      if (n == 0 && e == 0 && lane == 0) NM_STAMP(p.trace, 6);
       const int o_base = o0 + q * 32;
       float q_scale = 1.0f;
       const float q_lo = p.epi_relu ? 0.0f : -128.0f;
@@ -356,14 +369,17 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_tempty + 8u * buf, 0u));   // the leader's MMA warp waits for both CTAs
+      if (e == 0 && lane == 0) { if (n == 0) NM_STAMP(p.trace, 7); if (n + 1 == my_count) NM_STAMP(p.trace, 8); }
     }
     // the staging patches must outlive the stores' reads of them; the writes complete with the grid
     if (lane == 0) tma_store_wait_read();
+    if (e == 0 && lane == 0) { NM_STAMP(p.trace, 9); NM_STAMP_VAL(p.trace, 11, cyc_tfull); }
   }
 
   // neither CTA may free tensor memory or exit while its partner can still signal or read it
   tc_fence_before();
   cluster_sync_all();
+  if (threadIdx.x == 0) NM_STAMP(p.trace, 10);
   if (warp == 0) {
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
   }
@@ -476,6 +492,7 @@ nm_status launch_umma_pair(const SpmmArgs& a, bool* handled) {
   if (p.out_i8 && !p.epi_scale) return NM_ERR_INVALID_ARG;
   p.status = a.status;
   p.spin_limit = kSpinLimit;
+  p.trace = trace_buffer();
   p.w_fresh = a.w_fresh ? 1 : 0;
   p.tiles_o2 = ceil_div(w->O, 256);
   const int64_t items = (int64_t)p.tiles_o2 * ceil_div(a.T, pl.tile_t);
@@ -489,9 +506,9 @@ nm_status launch_umma_pair(const SpmmArgs& a, bool* handled) {
   if (!make_map(&tmB, a.X, (uint64_t)w->K * eb, (uint64_t)a.T, (uint64_t)a.ldx * eb, 128u, (uint32_t)pl.tile_t / 2u, true))
     return NM_ERR_CUDA;
   if (sp) {
-    // the metadata blocks as a 2-D tensor of 16-byte rows: one box = the blocks of one K step
-    const uint64_t rows = (uint64_t)ceil_div(w->O, kTileO) * w->hw24_meta_kblocks * 128u;
-    if (!make_map(&tmM, base + w->off_hw24_meta, 16u, rows, 16u, 16u, mb / 16u, false)) return NM_ERR_CUDA;
+    // the metadata blocks as a 2-D tensor of 2 KB rows: one box = the blocks of one K step
+    const uint64_t n_blocks = (uint64_t)ceil_div(w->O, kTileO) * w->hw24_meta_kblocks;
+    if (!make_meta_map(&tmM, base + w->off_hw24_meta, n_blocks, mb / 2048u)) return NM_ERR_CUDA;
   } else {
     tmM = tmB;
   }

@@ -38,6 +38,32 @@ __device__ __forceinline__ uint32_t requant_low_byte(uint32_t acc_bits, float sc
   return __float_as_uint(__fadd_rn(v, 12582912.0f));
 }
 
+// ------------------------------------------------------------------ phase stamps (trace builds only)
+// Compiled with -DNM_TRACE, every CTA of the tcgen05 kernels writes wall-clock stamps (%globaltimer,
+// nanoseconds, one clock for all SMs and all launches) of its pipeline phases into a caller buffer
+// of 16 x uint64 per CTA, set with nm_trace_set_buffer() before the call.  The normal build contains
+// none of this.  Slots: 0 kernel entry, 1 prologue done, 2 producer past the grid-dependency wait,
+// 3 first ring stage full (issuer), 4 first tile's last commit, 5 last tile's last commit,
+// 6 first accumulator ready (epilogue warp 2), 7 first tile's last store issued, 8 last tile's last
+// store issued, 9 staging patch free again, 10 about to free tensor memory, 12 tiles of this CTA;
+// SM cycles spent inside waits: 11 epilogue warp 2 for an accumulator, 13 issuing warp for a loaded
+// stage, 14 issuing warp for a drained accumulator, 15 producer for a free stage.
+#ifdef NM_TRACE
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// NM_WAIT_TIMED(acc, call): runs `call` (a bounded wait) and adds the SM cycles it took to `acc`
+#define NM_WAIT_TIMED(acc, call) do { const long long nm_t0_ = clock64(); call; (acc) += clock64() - nm_t0_; } while (0)
+#define NM_STAMP(buf, slot) do { if (buf) (buf)[(size_t)blockIdx.x * 16 + (slot)] = global_ns(); } while (0)
+#define NM_STAMP_VAL(buf, slot, v) do { if (buf) (buf)[(size_t)blockIdx.x * 16 + (slot)] = (unsigned long long)(v); } while (0)
+#else
+#define NM_WAIT_TIMED(acc, call) do { call; } while (0)
+#define NM_STAMP(buf, slot) do { } while (0)
+#define NM_STAMP_VAL(buf, slot, v) do { } while (0)
+#endif
+
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -72,7 +98,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
     if (i > 128) __nanosleep(64);
   }
   *w.abort_flag = 1u;
-  if (w.status) atomicOr(w.status, (uint32_t)NM_ERR_TIMEOUT | (site << 8));
+  if (w.status) atomicOr(w.status, (uint32_t)NM_ERR_TIMEOUT | (1u << (8u + site)));     // one bit per site: several may expire
   return false;
 }
 // The same poll without reporting: used on the way out of an aborted CTA to let copies that are
@@ -244,6 +270,22 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t r
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The 2:4 metadata blocks as a tensor of 2048-byte rows (256 elements of 8 bytes: the widest row a
+// tiled map can describe), box = the `rows_per_box` blocks of one K step.  A copy engine request
+// covers one row of the box, so rows of 16 bytes -- the natural row of a metadata block -- would
+// turn a 4 KB transfer into 256 requests; rows of 2 KB make it two.
+bool make_meta_map(CUtensorMap* map, const void* base, uint64_t n_blocks, uint32_t rows_per_box) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {256u, n_blocks};
+  cuuint64_t strides[1] = {2048u};
+  cuuint32_t box[2] = {256u, rows_per_box};
+  cuuint32_t estr[2] = {1u, 1u};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 uint32_t pow2_cols(uint32_t need) {
