@@ -34,7 +34,7 @@ def main():
     ap.add_argument("--cta-group", type=int, default=0)
     ap.add_argument("--issuers", type=int, default=0)
     ap.add_argument("--merge", default=None, choices=[None, "workspace", "cluster"], help="split-K merge (default: the planner's, or workspace under overrides)")
-    ap.add_argument("--path", default=None, choices=[None, "simt", "dense", "sp24", "decode", "expand"])
+    ap.add_argument("--path", default=None, choices=[None, "simt", "dense", "sp24", "decode", "expand", "remap"])
     ap.add_argument("--eager", action="store_true", help="time eager launches instead of one CUDA graph")
     ap.add_argument("--cublas", action="store_true", help="also time dense cuBLAS (torch._int_mm / torch.matmul) on the same buffers")
     ap.add_argument("--images", default="auto", choices=["auto", "all", "canonical"])
@@ -51,10 +51,14 @@ def main():
     if od is None:
         od = nm.NM_OUT_I32 if args.dtype == "i8" else nm.NM_OUT_F16
     images = {"auto": nm.NM_IMG_AUTO, "all": nm.NM_IMG_AUTO | nm.NM_IMG_DENSE | nm.NM_IMG_HW24, "canonical": nm.NM_IMG_CANONICAL}[args.images]
+    if args.path == "remap":
+        images |= nm.NM_IMG_REMAP48
     w = nm.nm_compress(W, n, m, images=images)
     plan = nm.nm_plan_create(args.T, w, od, 0)
     if args.path:
-        plan.path = {"simt": nm.NM_PATH_SIMT, "dense": nm.NM_PATH_UMMA_DENSE, "sp24": nm.NM_PATH_UMMA_SP24, "decode": nm.NM_PATH_UMMA_DECODE, "expand": nm.NM_PATH_UMMA_EXPAND}[args.path]
+        plan.path = {"simt": nm.NM_PATH_SIMT, "dense": nm.NM_PATH_UMMA_DENSE, "sp24": nm.NM_PATH_UMMA_SP24, "decode": nm.NM_PATH_UMMA_DECODE, "expand": nm.NM_PATH_UMMA_EXPAND, "remap": nm.NM_PATH_UMMA_REMAP48}[args.path]
+        if args.path == "remap":
+            plan.split_k, plan.cta_group, plan.resident = 1, 1, nm.NM_RES_NONE
         if args.path == "decode":
             plan.resident = nm.NM_RES_W
     if args.tile_t:
@@ -75,6 +79,8 @@ def main():
         plan.merge = nm.NM_MERGE_WORKSPACE
     t_pad = -(-args.T // plan.tile_t) * plan.tile_t
     plan.workspace_bytes = 0 if (plan.split_k <= 1 or plan.merge == nm.NM_MERGE_CLUSTER) else plan.split_k * t_pad * args.O * 4
+    if plan.path == nm.NM_PATH_UMMA_REMAP48:         # the gathered third-chunk activations sit at the head of the workspace
+        plan.workspace_bytes = -(-(args.T * (-(-(args.K // 2 * (1 if args.dtype == "i8" else 2)) // 16) * 16)) // 256) * 256
     if plan.path == nm.NM_PATH_UMMA_EXPAND:          # the dense copy sits at the head of the workspace
         plan.workspace_bytes += -(-(args.O * (-(-(args.K * (1 if args.dtype == "i8" else 2)) // 16) * 16)) // 256) * 256
 

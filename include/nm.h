@@ -61,6 +61,8 @@ enum {
   NM_IMG_HW24 = 2u,      /* 2:4-compressed values + hardware metadata blocks; exists when
                             every 4-chunk of W holds <= 2 nonzeros (always for n<=2, 4|m) */
   NM_IMG_DENSE = 4u,     /* W~ itself, row pitch rounded to 16 B (n==m reuses canonical)  */
+  NM_IMG_REMAP48 = 8u,   /* three-chunk K remap (see NM_PATH_UMMA_REMAP48): exists when every aligned
+                            group of 8 k holds <= 4 nonzeros (4:8, 3:8, ...); only built on request */
   NM_IMG_AUTO = 0x80000000u /* let nm_compress choose everything that applies            */
 };
 
@@ -71,13 +73,25 @@ enum {
   NM_PATH_UMMA_SP24 = 2,  /* TMA -> smem -> tcgen05.mma.sp (2:4 hardware sparsity)         */
   NM_PATH_UMMA_DECODE = 3,/* canonical image -> decode warps build the zero-filled micro-dense
                              tile in smem -> dense tcgen05.mma; any n:m, no extra image   */
-  NM_PATH_UMMA_EXPAND = 4 /* canonical image -> one small kernel writes the zero-filled dense rows
+  NM_PATH_UMMA_EXPAND = 4,/* canonical image -> one small kernel writes the zero-filled dense rows
                              once into the head of the workspace (O x round_up(K*eb,16) bytes,
                              counted in nm_plan.workspace_bytes; it stays in L2) -> the dense
                              tcgen05.mma path reads it.  For token counts where decoding the same
                              W tile again for every token tile would dominate; any n:m, no extra
                              image.  Without enough workspace an automatic plan falls back to
                              NM_PATH_UMMA_DECODE                                          */
+  NM_PATH_UMMA_REMAP48 = 5 /* 4:8-type weights on the 2:4 sparse tensor core at 3/4 of the dense MMA
+                             count.  A group of 8 k with up to 4 nonzeros is spread over THREE 4-chunks of
+                             a longer K axis, each holding <= 2: the two chunks of the group itself, and a
+                             third one that repeats the activations k+0, k+1, k+4, k+5 of the group and
+                             takes whatever a chunk holds beyond two (any 3 of 4 positions include one of
+                             the first two, so the move is always possible).  The third chunks of all
+                             groups form an extra K range of K/2, whose activations one small kernel
+                             gathers into the head of the workspace (T x round_up(K/2*eb,16) bytes) before
+                             the sparse kernel runs over K + K/2.  Opt-in (nm_plan_create never selects
+                             it): it needs NM_IMG_REMAP48, single CTAs, no split-K; it loads 1.5x the
+                             activation bytes and measured slower than the dense path on B200, whose
+                             tcgen05 kernels are bound by operand movement, not by MMA count               */
 };
 
 /* Operand residency of the tcgen05 paths (nm_plan.resident).  A persistent CTA walks a
@@ -122,6 +136,12 @@ typedef struct nm_weight {
   uint64_t hw24_row_bytes, dense_row_bytes;            /* row pitches in bytes */
   int32_t hw24_meta_kblocks;                           /* 2 KB metadata blocks per 128-row tile */
   int32_t reserved;
+  /* NM_IMG_REMAP48 (0 when absent): a 2:4 image of the remapped weight W' [O x remap_k], whose columns
+   * [0, K) are W without the moved elements, [K, remap_k_main) zero padding up to a whole K step, and
+   * [remap_k_main, remap_k) the third chunks: column remap_k_main + 4g + j pairs with activation
+   * 8g + {0,1,4,5}[j] */
+  uint64_t off_remap_values, off_remap_meta, remap_row_bytes;
+  int32_t remap_meta_kblocks, remap_k, remap_k_main, reserved2;
 } nm_weight;
 
 /* Launch plan: a deterministic function of (T, O, K, n, m, dtypes, images, #SMs). */

@@ -20,8 +20,8 @@ NM_OK, NM_ERR_INVALID_ARG, NM_ERR_SHAPE, NM_ERR_ALIGN, NM_ERR_NOT_NM = 0, 1, 2, 
 NM_ERR_UNSUPPORTED, NM_ERR_WORKSPACE, NM_ERR_ARCH, NM_ERR_CUDA, NM_ERR_TIMEOUT = 5, 6, 7, 8, 9
 NM_I8, NM_F16 = 0, 1
 NM_OUT_I32, NM_OUT_F32, NM_OUT_F16, NM_OUT_I8 = 0, 1, 2, 3
-NM_IMG_CANONICAL, NM_IMG_HW24, NM_IMG_DENSE, NM_IMG_AUTO = 1, 2, 4, 0x80000000
-NM_PATH_SIMT, NM_PATH_UMMA_DENSE, NM_PATH_UMMA_SP24, NM_PATH_UMMA_DECODE, NM_PATH_UMMA_EXPAND = 0, 1, 2, 3, 4
+NM_IMG_CANONICAL, NM_IMG_HW24, NM_IMG_DENSE, NM_IMG_REMAP48, NM_IMG_AUTO = 1, 2, 4, 8, 0x80000000
+NM_PATH_SIMT, NM_PATH_UMMA_DENSE, NM_PATH_UMMA_SP24, NM_PATH_UMMA_DECODE, NM_PATH_UMMA_EXPAND, NM_PATH_UMMA_REMAP48 = 0, 1, 2, 3, 4, 5
 NM_RES_NONE, NM_RES_X, NM_RES_W = 0, 1, 2
 NM_MERGE_WORKSPACE, NM_MERGE_CLUSTER = 0, 1
 NM_PLAN_DIAG_STALL = 1
@@ -44,6 +44,9 @@ class NMWeight(ctypes.Structure):
         ("off_hw24_values", ctypes.c_uint64), ("off_hw24_meta", ctypes.c_uint64), ("off_dense", ctypes.c_uint64),
         ("hw24_row_bytes", ctypes.c_uint64), ("dense_row_bytes", ctypes.c_uint64),
         ("hw24_meta_kblocks", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("off_remap_values", ctypes.c_uint64), ("off_remap_meta", ctypes.c_uint64), ("remap_row_bytes", ctypes.c_uint64),
+        ("remap_meta_kblocks", ctypes.c_int32), ("remap_k", ctypes.c_int32), ("remap_k_main", ctypes.c_int32),
+        ("reserved2", ctypes.c_int32),
     ]
 
 

@@ -78,7 +78,7 @@ __attribute__((visibility("default"))) void nm_trace_set_buffer(void* dev_buf) {
 
 size_t nm_packed_size(int O, int K, int n, int m, nm_dtype dt, uint32_t images) {
   PackLayout L;
-  uint32_t img = (images & NM_IMG_AUTO) ? (NM_IMG_CANONICAL | NM_IMG_HW24 | NM_IMG_DENSE) : images;
+  uint32_t img = (images & NM_IMG_AUTO) ? (NM_IMG_CANONICAL | NM_IMG_HW24 | NM_IMG_DENSE | (images & NM_IMG_REMAP48)) : images;
   if (pack_layout(O, K, n, m, dt, img, &L) != NM_OK) return 0;
   return (size_t)L.bytes;
 }
@@ -111,6 +111,11 @@ static nm_status pack_to_host(const void* W, int64_t ldw, int O, int K, int n, i
     img = images | NM_IMG_CANONICAL;
     if ((img & NM_IMG_HW24) && !clean) return NM_ERR_UNSUPPORTED;
   }
+  // the K remap is only built on request, for weights it applies to (not dense, at most 4 nonzeros per 8 k)
+  if (images & NM_IMG_REMAP48) {
+    if (n == m || !is_48_remappable(W, ldw, O, K, dt)) return NM_ERR_UNSUPPORTED;
+    img |= NM_IMG_REMAP48;
+  }
   PackLayout L;
   st = pack_layout(O, K, n, m, dt, img, &L);
   if (st != NM_OK) return st;
@@ -124,6 +129,7 @@ static nm_status pack_to_host(const void* W, int64_t ldw, int O, int K, int n, i
   if (img & NM_IMG_HW24)
     build_hw24(W, ldw, O, K, dt, L, host + L.off_hw24_values, host + L.off_hw24_meta);
   if (L.off_dense) build_dense(W, ldw, O, K, dt, L, host + L.off_dense);
+  if (L.off_remap_values) build_remap48(W, ldw, O, K, dt, L, host + L.off_remap_values, host + L.off_remap_meta);
 
   std::memset(out, 0, sizeof(*out));
   out->magic = kWeightMagic; out->version = 1;
@@ -136,6 +142,10 @@ static nm_status pack_to_host(const void* W, int64_t ldw, int O, int K, int n, i
   out->off_dense = L.off_dense;
   out->hw24_row_bytes = L.hw24_row_bytes; out->dense_row_bytes = L.dense_row_bytes;
   out->hw24_meta_kblocks = L.hw24_meta_kblocks;
+  if (!L.off_remap_values) out->images &= ~(uint32_t)NM_IMG_REMAP48;
+  out->off_remap_values = L.off_remap_values; out->off_remap_meta = L.off_remap_meta;
+  out->remap_row_bytes = L.remap_row_bytes; out->remap_meta_kblocks = L.remap_meta_kblocks;
+  out->remap_k = L.remap_k; out->remap_k_main = L.remap_k_main;
   return NM_OK;
 }
 
@@ -283,6 +293,32 @@ nm_status nm_spmm_ex(const void* X, int64_t ldx, int T, const nm_weight* w, cons
       a.workspace = static_cast<uint8_t*>(workspace) + head;
       a.workspace_bytes = workspace_bytes - head;
     }
+  }
+  // NM_PATH_UMMA_REMAP48: gather the third-chunk activations into the head of the workspace, then run the
+  // sparse kernel over the remapped weight; its K steps beyond the main range read the gathered copy
+  nm_weight remapped;
+  if (a.plan.path == NM_PATH_UMMA_REMAP48) {
+    if (!(w->images & NM_IMG_REMAP48) || !w->off_remap_values) return NM_ERR_UNSUPPORTED;
+    if (a.plan.split_k > 1 || a.plan.resident != NM_RES_NONE || epi) return NM_ERR_INVALID_ARG;
+    const uint64_t head = remap_workspace_bytes(T, w->K, eb);
+    if (!workspace || workspace_bytes < head) return NM_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 15) return NM_ERR_ALIGN;
+    st = launch_remap_gather(X, ldx, T, w->K, w->dtype, workspace, stream);
+    if (st != NM_OK) return st;
+    remapped = *w;
+    remapped.K = w->remap_k; remapped.n = 2; remapped.m = 4;
+    remapped.images = NM_IMG_HW24;
+    remapped.off_hw24_values = w->off_remap_values; remapped.off_hw24_meta = w->off_remap_meta;
+    remapped.hw24_row_bytes = w->remap_row_bytes; remapped.hw24_meta_kblocks = w->remap_meta_kblocks;
+    a.w = &remapped;
+    a.X_ovf = workspace;
+    a.ld_ovf = (int64_t)(round_up((uint64_t)(w->K / 2) * eb, 16) / eb);
+    a.k_x = w->K; a.k_ovf = w->K / 2;
+    a.ksteps_main = w->remap_k_main * eb / 256;
+    a.plan.path = NM_PATH_UMMA_SP24;
+    a.plan.cta_group = 1;
+    a.workspace = static_cast<uint8_t*>(workspace) + head;
+    a.workspace_bytes = workspace_bytes - head;
   }
   switch (a.plan.path) {
     case NM_PATH_SIMT: return launch_simt(a);

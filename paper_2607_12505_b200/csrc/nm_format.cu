@@ -49,6 +49,21 @@ nm_status pack_layout(int O, int K, int n, int m, int dt, uint32_t images, PackL
     L->off_dense = off;
     off = round_up(off + (uint64_t)O * L->dense_row_bytes, 256);
   }
+  L->off_remap_values = L->off_remap_meta = L->remap_row_bytes = L->remap_meta_bytes = 0;
+  L->remap_meta_kblocks = L->remap_k = L->remap_k_main = 0;
+  if ((images & NM_IMG_REMAP48) && n != m && K % 8 == 0) {
+    // W' = [W without the moved elements | zero padding to a whole K step | third chunks (K/2 columns)]
+    const int step_elems = 256 / eb;                       // logical k of one sparse K step (256 B of activations)
+    L->remap_k_main = ceil_div(K, step_elems) * step_elems;
+    L->remap_k = L->remap_k_main + K / 2;
+    L->remap_row_bytes = round_up((uint64_t)(L->remap_k / 4) * 2 * eb, 16);
+    L->off_remap_values = off;
+    off = round_up(off + (uint64_t)O * L->remap_row_bytes, 256);
+    L->remap_meta_kblocks = (dt == NM_I8) ? 2 * ceil_div(L->remap_k, 256) : ceil_div(L->remap_k, 128);
+    L->remap_meta_bytes = (uint64_t)ceil_div(O, kTileO) * L->remap_meta_kblocks * kMetaBlockBytes;
+    L->off_remap_meta = off;
+    off = round_up(off + L->remap_meta_bytes, 256);
+  }
   L->bytes = off;
   return NM_OK;
 }
@@ -176,6 +191,59 @@ void build_hw24(const void* W, int64_t ldw, int O, int K, int dt, const PackLayo
     }
   }
   (void)eb;
+}
+
+bool is_48_remappable(const void* W, int64_t ldw, int O, int K, int dt) {
+  if (K % 8 != 0) return false;
+  for (int o = 0; o < O; ++o)
+    for (int g = 0; g < K / 8; ++g) {
+      int cnt = 0;
+      for (int p = 0; p < 8; ++p) cnt += !elem_is_zero(W, dt, (int64_t)o * ldw + g * 8 + p);
+      if (cnt > 4) return false;
+    }
+  return true;
+}
+
+// Three-chunk K remap (NM_PATH_UMMA_REMAP48).  For every row and group of 8 k: a 4-chunk that holds
+// more than two nonzeros hands the excess to the group's third chunk, taking it from its first two
+// positions (k+0, k+1 of the first chunk; k+4, k+5 of the second), which are the ones the third chunk
+// repeats; any three of four positions include one of the first two, all four include both, and a
+// group with at most 4 nonzeros has an excess of at most two.  The remapped row is then 2:4-clean and
+// is packed by the ordinary 2:4 packer.
+void build_remap48(const void* W, int64_t ldw, int O, int K, int dt, const PackLayout& L, uint8_t* values, uint8_t* meta) {
+  const int eb = elem_bytes(dt);
+  const int Kr = L.remap_k, Km = L.remap_k_main;
+  std::vector<uint8_t> Wr((size_t)O * Kr * eb, 0);
+  auto get = [&](int o, int k) -> uint16_t {
+    return dt == NM_I8 ? (uint16_t)(uint8_t)static_cast<const int8_t*>(W)[(int64_t)o * ldw + k]
+                       : static_cast<const uint16_t*>(W)[(int64_t)o * ldw + k];
+  };
+  auto put = [&](int o, int k, uint16_t v) {
+    if (dt == NM_I8) Wr[(size_t)o * Kr + k] = (uint8_t)v;
+    else reinterpret_cast<uint16_t*>(Wr.data())[(size_t)o * Kr + k] = v;
+  };
+  for (int o = 0; o < O; ++o)
+    for (int g = 0; g < K / 8; ++g)
+      for (int half = 0; half < 2; ++half) {
+        const int k0 = g * 8 + half * 4;
+        int nz = 0;
+        for (int p = 0; p < 4; ++p) nz += !elem_is_zero(W, dt, (int64_t)o * ldw + k0 + p);
+        int excess = nz > 2 ? nz - 2 : 0;
+        for (int p = 0; p < 4; ++p) {
+          const bool zero = elem_is_zero(W, dt, (int64_t)o * ldw + k0 + p);
+          if (!zero && excess > 0 && p < 2) {          // moved to the third chunk: slot 2*half + p
+            put(o, Km + g * 4 + half * 2 + p, get(o, k0 + p));
+            --excess;
+          } else if (!zero) {
+            put(o, k0 + p, get(o, k0 + p));
+          }
+        }
+      }
+  PackLayout T = L;                                    // the 2:4 packer reads its geometry from these fields
+  T.hw24_row_bytes = L.remap_row_bytes;
+  T.hw24_meta_kblocks = L.remap_meta_kblocks;
+  T.hw24_meta_bytes = L.remap_meta_bytes;
+  build_hw24(Wr.data(), Kr, O, Kr, dt, T, values, meta);
 }
 
 void build_dense(const void* W, int64_t ldw, int O, int K, int dt, const PackLayout& L, uint8_t* dense) {

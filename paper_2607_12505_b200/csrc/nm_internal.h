@@ -37,6 +37,9 @@ struct PackLayout {
   uint64_t hw24_row_bytes, dense_row_bytes;
   int hw24_meta_kblocks;        // 2 KB blocks along K per 128-row tile
   uint64_t hw24_meta_bytes;
+  // three-chunk K remap image (NM_IMG_REMAP48): a 2:4 image of W' [O x remap_k]
+  uint64_t off_remap_values, off_remap_meta, remap_row_bytes, remap_meta_bytes;
+  int remap_meta_kblocks, remap_k, remap_k_main;
   uint64_t bytes;
 };
 nm_status pack_layout(int O, int K, int n, int m, int dt, uint32_t images, PackLayout* L);
@@ -49,6 +52,9 @@ void build_hw24(const void* W, int64_t ldw, int O, int K, int dt, const PackLayo
                 uint8_t* values, uint8_t* meta);
 void build_dense(const void* W, int64_t ldw, int O, int K, int dt, const PackLayout& L, uint8_t* dense);
 nm_status decode_canonical(const uint8_t* canon, size_t bytes, void* W, int64_t ldw);
+// NM_IMG_REMAP48: true when every aligned group of 8 k holds at most 4 nonzeros (K % 8 == 0)
+bool is_48_remappable(const void* W, int64_t ldw, int O, int K, int dt);
+void build_remap48(const void* W, int64_t ldw, int O, int K, int dt, const PackLayout& L, uint8_t* values, uint8_t* meta);
 
 // ---- kernel launchers (nm_kernels_*.cu) ----------------------------------------------
 struct SpmmArgs {
@@ -60,12 +66,18 @@ struct SpmmArgs {
   uint32_t* status;
   void* stream;
   nm_epilogue epi;         // scale_dev == nullptr: no epilogue
+  // NM_PATH_UMMA_REMAP48: K steps below ksteps_main read X, the others the gathered third-chunk activations
+  const void* X_ovf = nullptr; int64_t ld_ovf = 0; int k_x = 0, k_ovf = 0, ksteps_main = 0;
   bool w_fresh = false;    // the weight image is written by the launch just before (no load ahead of the grid-dependency wait)
 };
 // NM_PATH_UMMA_EXPAND: bytes of the dense copy at the head of the workspace (256-byte multiple)
 uint64_t expand_workspace_bytes(int O, int K, int eb);
 // enqueues the expansion of the canonical image into `dst` (rows of round_up(K*eb,16) bytes)
 nm_status launch_expand(const nm_weight* w, void* dst, void* stream);
+// NM_PATH_UMMA_REMAP48: bytes of the gathered activations at the head of the workspace, and the gather itself
+// (dst[t, 4g + j] = X[t, 8g + {0,1,4,5}[j]], rows of round_up(K/2*eb, 16) bytes)
+uint64_t remap_workspace_bytes(int T, int K, int eb);
+nm_status launch_remap_gather(const void* X, int64_t ldx, int T, int K, int dt, void* dst, void* stream);
 nm_status launch_simt(const SpmmArgs& a);
 nm_status launch_umma(const SpmmArgs& a);
 nm_status launch_umma_pair(const SpmmArgs& a, bool* handled);   // cta_group::2 variant; may decline

@@ -190,6 +190,55 @@ uint64_t expand_workspace_bytes(int O, int K, int eb) {
   return round_up((uint64_t)O * round_up((uint64_t)K * eb, 16), 256);
 }
 
+// Gather of the third-chunk activations of the 4:8 K remap (NM_PATH_UMMA_REMAP48): for every token row
+// and group of 8 k, the elements k+0, k+1, k+4, k+5.  One thread per group: one 8- or 16-byte load,
+// one 4- or 8-byte store.  X may come from the launch before, so it is read after the dependency wait.
+template <int EB>
+__global__ void __launch_bounds__(256)
+nm_remap_gather_kernel(const uint8_t* __restrict__ X, int64_t x_pitch, int T, int G8, uint8_t* __restrict__ dst, int64_t dst_pitch) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int64_t total = (int64_t)T * G8;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int t = (int)(i / G8), g = (int)(i % G8);
+    if (EB == 1) {
+      const uint2 v = *reinterpret_cast<const uint2*>(X + (int64_t)t * x_pitch + (int64_t)g * 8);
+      *reinterpret_cast<uint32_t*>(dst + (int64_t)t * dst_pitch + (int64_t)g * 4) = (v.x & 0xffffu) | (v.y << 16);
+    } else {
+      const uint4 v = *reinterpret_cast<const uint4*>(X + (int64_t)t * x_pitch + (int64_t)g * 16);
+      *reinterpret_cast<uint2*>(dst + (int64_t)t * dst_pitch + (int64_t)g * 8) = make_uint2(v.x, v.z);
+    }
+  }
+}
+
+uint64_t remap_workspace_bytes(int T, int K, int eb) {
+  return round_up((uint64_t)T * round_up((uint64_t)(K / 2) * eb, 16), 256);
+}
+
+nm_status launch_remap_gather(const void* X, int64_t ldx, int T, int K, int dt, void* dst, void* stream) {
+  const int eb = elem_bytes(dt);
+  const int G8 = K / 8;
+  const int64_t total = (int64_t)T * G8;
+  cudaLaunchConfig_t cfg = {};
+  int64_t blocks = (total + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  cfg.gridDim = dim3((unsigned)(blocks < 1 ? 1 : blocks));
+  cfg.blockDim = dim3(256);
+  cfg.stream = static_cast<cudaStream_t>(stream);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const int64_t x_pitch = ldx * eb, d_pitch = (int64_t)round_up((uint64_t)(K / 2) * eb, 16);
+  const cudaError_t e = dt == NM_I8
+      ? cudaLaunchKernelEx(&cfg, nm_remap_gather_kernel<1>, static_cast<const uint8_t*>(X), x_pitch, T, G8, static_cast<uint8_t*>(dst), d_pitch)
+      : cudaLaunchKernelEx(&cfg, nm_remap_gather_kernel<2>, static_cast<const uint8_t*>(X), x_pitch, T, G8, static_cast<uint8_t*>(dst), d_pitch);
+  if (e != cudaSuccess) { cudaGetLastError(); return NM_ERR_CUDA; }
+  count_launch();
+  return NM_OK;
+}
+
 nm_status launch_expand(const nm_weight* w, void* dst, void* stream) {
   CanonGeom g;
   nm_status st = canon_geom(w->O, w->K, w->n, w->m, w->dtype, &g);

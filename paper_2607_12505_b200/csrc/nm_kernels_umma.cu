@@ -63,6 +63,8 @@ struct UmmaParams {
   int acc_bufs;             // TMEM accumulator buffers (2 when 2*tile_t + metadata fit in 512 columns)
   int tiles_o, n_items;     // out-feature tiles; work items = tiles * split_k
   int total_ksteps;         // K steps of 128 B of A per row
+  int ksteps_main;          // K remap (NM_PATH_UMMA_REMAP48): K steps from this one on read the gathered third-chunk
+                            // activations through the second X map (>= total_ksteps: no remap)
   int ksteps_per_split, split_k;
   int out_f16;              // fp16 path: 1 = convert to half on store
   int out_i8;               // int8 path with requantising epilogue: 1 = scale / bias / ReLU / saturate to int8
@@ -301,7 +303,7 @@ __device__ __forceinline__ void decode_row_kstep(const UmmaParams& p, uint32_t t
 template <int DT, bool SP, bool DEC, bool DUAL, bool CLU>
 __global__ void __launch_bounds__(DEC ? kThreadsDec : kThreads + 32, 1)      // the decode warps only exist in the DEC variants
 nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmY, const UmmaParams p) {
+               const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY, const UmmaParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -330,6 +332,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     pdl_launch_dependents();
     prefetch_tensormap(&tmA);
     prefetch_tensormap(&tmB);
+    if (SP && p.ksteps_main < p.total_ksteps) prefetch_tensormap(&tmB2);
     if (p.epi_mode == kEpiTma) prefetch_tensormap(&tmY);
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(bar_full + 8u * s, (DEC && p.resident != NM_RES_W) ? 1 + kDecWarps : 1);
@@ -393,8 +396,12 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // that the first real loads after the wait do not pay the HBM latency
         for (int i = 0; i < pre; ++i) {
           if (SP) {
-            tma_prefetch_l2_2d(&tmB, (c0.ks_begin + i) * 256, c0.t0);
-            tma_prefetch_l2_2d(&tmB, (c0.ks_begin + i) * 256 + 128, c0.t0);
+            const int ks = c0.ks_begin + i;
+            const bool ovf = ks >= p.ksteps_main;
+            const CUtensorMap* bm = ovf ? &tmB2 : &tmB;
+            const int kx = (ovf ? ks - p.ksteps_main : ks) * 256;
+            tma_prefetch_l2_2d(bm, kx, c0.t0);
+            tma_prefetch_l2_2d(bm, kx + 128, c0.t0);
           } else {
             tma_prefetch_l2_2d(&tmB, (c0.ks_begin + i) * 128, c0.t0);
           }
@@ -405,7 +412,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       NM_STAMP_VAL(p.trace, 12, R.count);
       uint32_t rloads = 0, s = 0, ph = 0, st = ring_base;
       uint32_t armed = 0;          // ring stages armed so far (K steps whose loads were issued)
-      long long cyc_empty = 0;     // trace builds: cycles spent waiting for a free stage
+      [[maybe_unused]] long long cyc_empty = 0;     // trace builds: cycles spent waiting for a free stage
       bool wrapped = false;
       int prev_key = -1;
       bool ok = true;
@@ -455,8 +462,12 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_expect_tx(full, ((DEC && p.resident != NM_RES_W) ? sbytes - 16384u : sbytes) + extra);   // decoded A is not a TMA transfer
           if (p.resident != NM_RES_X) {            // B part streams
             if (SP) {
-              tma_load_2d(st, &tmB, full, ks * 256, c.t0);
-              tma_load_2d(st + b_tile_bytes, &tmB, full, ks * 256 + 128, c.t0);
+              // under the K remap the K steps of the third chunks read their activations from the gathered copy
+              const bool ovf = ks >= p.ksteps_main;
+              const CUtensorMap* bm = ovf ? &tmB2 : &tmB;
+              const int kx = (ovf ? ks - p.ksteps_main : ks) * 256;
+              tma_load_2d(st, bm, full, kx, c.t0);
+              tma_load_2d(st + b_tile_bytes, bm, full, kx + 128, c.t0);
             } else {
               tma_load_2d(st, &tmB, full, ks * 128, c.t0);
             }
@@ -513,7 +524,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       bool ok = true;
       ItemWalker walk;
       walk.init(p, R);
-      long long cyc_full = 0, cyc_tempty = 0;      // trace builds: cycles spent inside the two waits of this warp
+      [[maybe_unused]] long long cyc_full = 0, cyc_tempty = 0;      // trace builds: cycles spent inside the two waits of this warp
       // The producer is parked behind the previous grid of the stream until that grid has finished;
       // waiting here too keeps that time out of this warp's bounded waits (it costs nothing once the
       // producer is through).
@@ -607,7 +618,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int ob = (DT == NM_F16 && p.out_f16 && !ws_split) ? 2 : ((DT == NM_I8 && p.out_i8 && !ws_split) ? 1 : 4);
     const uint32_t crank = CLU ? cluster_cta_rank() : 0u;
     const ItemRange R = my_items(p);
-    long long cyc_tfull = 0;      // trace builds: cycles spent waiting for an accumulator
+    [[maybe_unused]] long long cyc_tfull = 0;      // trace builds: cycles spent waiting for an accumulator
     pdl_wait_prior_grid();        // Y / workspace may still be in use by the previous kernel
     for (int n = 0; n < R.count; ++n) {
       const uint32_t li = (uint32_t)n;
@@ -864,7 +875,7 @@ nm_status launch_merge(const SpmmArgs& a, const UmmaParams& p) {
 
 // one instantiation of the kernel: shared-memory opt-in once per device, then the launch
 template <int DT, bool SP, bool DEC, bool DUAL, bool CLU>
-nm_status launch_variant(const cudaLaunchConfig_t& cfg, const CUtensorMap& tmA, const CUtensorMap& tmB,
+nm_status launch_variant(const cudaLaunchConfig_t& cfg, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2,
                          const CUtensorMap& tmY, const UmmaParams& p) {
   static std::atomic<uint64_t> configured{0};        // the attribute belongs to the (function, device) pair
   const int slot = device_slot();
@@ -873,7 +884,7 @@ nm_status launch_variant(const cudaLaunchConfig_t& cfg, const CUtensorMap& tmA, 
       return NM_ERR_CUDA;
     configured.fetch_or(1ull << slot, std::memory_order_relaxed);
   }
-  if (cudaLaunchKernelEx(&cfg, nm_umma_kernel<DT, SP, DEC, DUAL, CLU>, tmA, tmB, tmY, p) != cudaSuccess) {
+  if (cudaLaunchKernelEx(&cfg, nm_umma_kernel<DT, SP, DEC, DUAL, CLU>, tmA, tmB, tmB2, tmY, p) != cudaSuccess) {
     cudaGetLastError();
     return NM_ERR_CUDA;
   }
@@ -881,7 +892,7 @@ nm_status launch_variant(const cudaLaunchConfig_t& cfg, const CUtensorMap& tmA, 
 }
 
 template <int DT, bool SP, bool DEC>
-nm_status launch_one(const SpmmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+nm_status launch_one(const SpmmArgs& a, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const CUtensorMap& tmY,
                      UmmaParams& p) {
   // Residency is a request: it needs every K step of the resident operand plus at least two
   // ring stages in shared memory, the metadata of a resident W in 64 TMEM columns, and no
@@ -943,11 +954,11 @@ nm_status launch_one(const SpmmArgs& a, const CUtensorMap& tmA, const CUtensorMa
   }
   nm_status lst;
   if (!DEC && p.cluster_merge)
-    lst = p.issuers == 2 ? launch_variant<DT, SP, false, true, true>(cfg, tmA, tmB, tmY, p)
-                         : launch_variant<DT, SP, false, false, true>(cfg, tmA, tmB, tmY, p);
+    lst = p.issuers == 2 ? launch_variant<DT, SP, false, true, true>(cfg, tmA, tmB, tmB2, tmY, p)
+                         : launch_variant<DT, SP, false, false, true>(cfg, tmA, tmB, tmB2, tmY, p);
   else
-    lst = (!DEC && p.issuers == 2) ? launch_variant<DT, SP, false, true, false>(cfg, tmA, tmB, tmY, p)
-                                   : launch_variant<DT, SP, DEC, false, false>(cfg, tmA, tmB, tmY, p);
+    lst = (!DEC && p.issuers == 2) ? launch_variant<DT, SP, false, true, false>(cfg, tmA, tmB, tmB2, tmY, p)
+                                   : launch_variant<DT, SP, DEC, false, false>(cfg, tmA, tmB, tmB2, tmY, p);
   if (lst != NM_OK) return lst;
   count_launch();
   return cudaGetLastError() == cudaSuccess ? NM_OK : NM_ERR_CUDA;
@@ -1003,6 +1014,8 @@ nm_status launch_umma(const SpmmArgs& a) {
   p.issuers = pl.issuers == 2 ? 2 : 1;
   p.w_fresh = a.w_fresh ? 1 : 0;
   p.total_ksteps = (int)((a_row_bytes + 127) / 128);
+  p.ksteps_main = a.X_ovf ? a.ksteps_main : 0x7fffffff;
+  if (a.X_ovf && (!sp || pl.split_k > 1 || pl.resident != NM_RES_NONE)) return NM_ERR_INVALID_ARG;
   int split = pl.split_k < p.total_ksteps ? pl.split_k : p.total_ksteps;
   p.ksteps_per_split = ceil_div(p.total_ksteps, split);
   split = ceil_div(p.total_ksteps, p.ksteps_per_split);         // no empty slice
@@ -1051,10 +1064,19 @@ nm_status launch_umma(const SpmmArgs& a) {
   const bool y_tma_ok = !(reinterpret_cast<uintptr_t>(y_base) & 15) && y_pitch % 16 == 0;
   p.epi_mode = y_tma_ok ? kEpiTma : ((split > 1 && !p.cluster_merge) ? kEpiSplit : kEpiDirect);
 
-  CUtensorMap tmA, tmB, tmY;
+  CUtensorMap tmA, tmB, tmB2, tmY;
   if (!dec && !make_map(&tmA, a_ptr, a_row_bytes, (uint64_t)w->O, a_pitch, 128u, kTileO, true)) return NM_ERR_CUDA;
-  if (!make_map(&tmB, a.X, (uint64_t)w->K * eb, (uint64_t)a.T, (uint64_t)a.ldx * eb, 128u, (uint32_t)pl.tile_t, true))
+  // under the K remap X keeps its own K columns (bytes beyond them read as zero: the padding of the main range)
+  // and the second map covers the gathered third-chunk activations
+  const uint64_t x_row_bytes = (uint64_t)(a.X_ovf ? a.k_x : w->K) * eb;
+  if (!make_map(&tmB, a.X, x_row_bytes, (uint64_t)a.T, (uint64_t)a.ldx * eb, 128u, (uint32_t)pl.tile_t, true))
     return NM_ERR_CUDA;
+  if (a.X_ovf) {
+    if (!make_map(&tmB2, a.X_ovf, (uint64_t)a.k_ovf * eb, (uint64_t)a.T, (uint64_t)a.ld_ovf * eb, 128u, (uint32_t)pl.tile_t, true))
+      return NM_ERR_CUDA;
+  } else {
+    tmB2 = tmB;
+  }
   if (dec) tmA = tmB;      // the decode path never loads W through TMA
   if (p.epi_mode == kEpiTma) {
     if (!make_map(&tmY, y_base, y_row_bytes, y_rows, y_pitch, y_box_bytes, 32u, false)) return NM_ERR_CUDA;
@@ -1064,11 +1086,11 @@ nm_status launch_umma(const SpmmArgs& a) {
 
   nm_status st;
   if (w->dtype == NM_I8) {
-    st = sp ? launch_one<NM_I8, true, false>(a, tmA, tmB, tmY, p)
-            : (dec ? launch_one<NM_I8, false, true>(a, tmA, tmB, tmY, p) : launch_one<NM_I8, false, false>(a, tmA, tmB, tmY, p));
+    st = sp ? launch_one<NM_I8, true, false>(a, tmA, tmB, tmB2, tmY, p)
+            : (dec ? launch_one<NM_I8, false, true>(a, tmA, tmB, tmB2, tmY, p) : launch_one<NM_I8, false, false>(a, tmA, tmB, tmB2, tmY, p));
   } else {
-    st = sp ? launch_one<NM_F16, true, false>(a, tmA, tmB, tmY, p)
-            : (dec ? launch_one<NM_F16, false, true>(a, tmA, tmB, tmY, p) : launch_one<NM_F16, false, false>(a, tmA, tmB, tmY, p));
+    st = sp ? launch_one<NM_F16, true, false>(a, tmA, tmB, tmB2, tmY, p)
+            : (dec ? launch_one<NM_F16, false, true>(a, tmA, tmB, tmB2, tmY, p) : launch_one<NM_F16, false, false>(a, tmA, tmB, tmB2, tmY, p));
   }
   if (st != NM_OK || split <= 1 || p.cluster_merge) return st;
   return w->dtype == NM_I8 ? launch_merge<NM_I8>(a, p) : launch_merge<NM_F16>(a, p);

@@ -168,35 +168,16 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // ---------------- TMA producer (both CTAs): own W rows, own half of the token tile
       // W tiles of the first ring-full of K steps are requested before the grid-dependency wait
       // (the packed weight never depends on the previous kernel); X only after it.
+      // (they are requested by warp 1, which has nothing else to do yet: this thread goes straight to the
+      // wait, so a CTA that starts after the previous grid has finished asks for X at once)
       const int pre = (my_count > 0 && !p.w_fresh) ? min(p.stages, p.total_ksteps) : 0;
-      for (int i = 0; i < pre; ++i) {
-        const int o0p = (pair % p.tiles_o2) * 256 + (int)rank * 128;
-        const uint32_t full_leader = map_to_cta(bar_full + 8u * (uint32_t)i, 0u);
-        const uint32_t sa = smem_base + (uint32_t)i * sbytes;
-        if (rank == 0u) mbar_expect_tx(bar_full + 8u * (uint32_t)i, 2u * sbytes);
-        tma_load_2d_pair(sa, &tmA, full_leader, i * 128, o0p);
-        if (SP) tma_load_2d_pair(sa + 16384u, &tmM, full_leader, 0,
-                                 ((o0p / kTileO) * p.total_ksteps + i) * (int)(meta_bytes2<DT, SP>() / 2048u));
-      }
-      // the X boxes of those K steps are pulled towards L2 (a hint, no data is consumed), so that
-      // the first real loads after the wait do not pay the HBM latency
-      for (int i = 0; i < pre; ++i) {
-        const int tile0p = (pair / p.tiles_o2) * p.tile_t, n_leftp = p.T - tile0p;
-        const int t0p = tile0p + (int)rank * ((n_leftp >= p.tile_t ? p.tile_t : ((n_leftp + 31) & ~31)) / 2);
-        if (SP) {
-          tma_prefetch_l2_2d(&tmB, i * 256, t0p);
-          tma_prefetch_l2_2d(&tmB, i * 256 + 128, t0p);
-        } else {
-          tma_prefetch_l2_2d(&tmB, i * 128, t0p);
-        }
-      }
       pdl_wait_prior_grid();
       NM_STAMP(p.trace, 2);
       NM_STAMP_VAL(p.trace, 12, my_count);
       bool ok = true, wrapped = false;
       // ring position kept incrementally (stage s, phase parity ph): no divisions in a lone thread
       uint32_t s = 0, ph = 0, sa = smem_base, armed = 0;
-      long long cyc_empty = 0;     // trace builds: cycles spent waiting for a free stage
+      [[maybe_unused]] long long cyc_empty = 0;     // trace builds: cycles spent waiting for a free stage
       for (int n = 0; n < my_count && ok; ++n) {
         const int item = pair + n * n_pairs;
         const int o0 = (item % p.tiles_o2) * 256 + (int)rank * 128;
@@ -244,6 +225,34 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
     }
   } else if (warp == 1) {
+    if (lane == 0) {
+      // Weight prefetch ahead of the grid-dependency wait (both CTAs, each its own W rows): the W
+      // tiles and metadata of the first ring-full of K steps; the leader arms the barriers with the
+      // byte count of the whole stage of both CTAs, the producers add the X tiles after their wait.
+      const int pre = (my_count > 0 && !p.w_fresh) ? min(p.stages, p.total_ksteps) : 0;
+      for (int i = 0; i < pre; ++i) {
+        const int o0p = (pair % p.tiles_o2) * 256 + (int)rank * 128;
+        const uint32_t full_leader = map_to_cta(bar_full + 8u * (uint32_t)i, 0u);
+        const uint32_t sa = smem_base + (uint32_t)i * sbytes;
+        if (rank == 0u) mbar_expect_tx(bar_full + 8u * (uint32_t)i, 2u * sbytes);
+        tma_load_2d_pair(sa, &tmA, full_leader, i * 128, o0p);
+        if (SP) tma_load_2d_pair(sa + 16384u, &tmM, full_leader, 0,
+                                 ((o0p / kTileO) * p.total_ksteps + i) * (int)(meta_bytes2<DT, SP>() / 2048u));
+      }
+      // the X boxes of those K steps are pulled towards L2 (a hint, no data is consumed), so that
+      // the first real loads after the wait do not pay the HBM latency
+      for (int i = 0; i < pre; ++i) {
+        const int tile0p = (pair / p.tiles_o2) * p.tile_t, n_leftp = p.T - tile0p;
+        const int t0p = tile0p + (int)rank * ((n_leftp >= p.tile_t ? p.tile_t : ((n_leftp + 31) & ~31)) / 2);
+        if (SP) {
+          tma_prefetch_l2_2d(&tmB, i * 256, t0p);
+          tma_prefetch_l2_2d(&tmB, i * 256 + 128, t0p);
+        } else {
+          tma_prefetch_l2_2d(&tmB, i * 128, t0p);
+        }
+      }
+    }
+    __syncwarp();
     if (rank == 0u) {
       // ---------------- MMA issuer (leader only): M = 256 across the pair, N = tile_t.  The whole
       // warp walks the loop in lockstep; the tcgen05 wrappers elect the lane that issues.
@@ -257,7 +266,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       // token-tile index of this pair's items, advanced without a division per item
       const int step_t = n_pairs / p.tiles_o2, step_o = n_pairs % p.tiles_o2;
       int t_idx = pair / p.tiles_o2, o_idx = pair % p.tiles_o2;
-      long long cyc_full = 0, cyc_tempty = 0;      // trace builds: cycles spent inside the two waits of this warp
+      [[maybe_unused]] long long cyc_full = 0, cyc_tempty = 0;      // trace builds: cycles spent inside the two waits of this warp
       pdl_wait_prior_grid();      // keeps the previous grid's run time out of the bounded waits below
       for (int n = 0; n < my_count && ok; ++n) {
         const uint32_t buf = (uint32_t)n % (uint32_t)p.acc_bufs, use = (uint32_t)n / (uint32_t)p.acc_bufs;
@@ -314,7 +323,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int e = warp - 2, q = warp & 3, h = e >> 2;
     const uint32_t patch = patches + (uint32_t)e * kPatchBytes2;
     const int ob = (DT == NM_F16 && p.out_f16) ? 2 : ((DT == NM_I8 && p.out_i8) ? 1 : 4);
-    long long cyc_tfull = 0;      // trace builds: cycles spent waiting for an accumulator
+    [[maybe_unused]] long long cyc_tfull = 0;      // trace builds: cycles spent waiting for an accumulator
     pdl_wait_prior_grid();
     for (int n = 0; n < my_count; ++n) {
       const int item = pair + n * n_pairs;

@@ -34,6 +34,10 @@ def make_plan(T, w, od, **over):
     t_pad = -(-T // plan.tile_t) * plan.tile_t               # slices hold whole token tiles
     on_chip = plan.merge == nm.NM_MERGE_CLUSTER
     plan.workspace_bytes = 0 if (plan.split_k <= 1 or on_chip or plan.path == nm.NM_PATH_SIMT) else plan.split_k * t_pad * w.desc.O * 4
+    if plan.path == nm.NM_PATH_UMMA_REMAP48:                 # the gathered third-chunk activations sit at the head
+        eb = 1 if w.desc.dtype == nm.NM_I8 else 2
+        plan.workspace_bytes = -(-(T * (-(-(w.desc.K // 2 * eb) // 16) * 16)) // 256) * 256
+        plan.split_k, plan.cta_group, plan.resident = 1, 1, nm.NM_RES_NONE
     if plan.path == nm.NM_PATH_UMMA_EXPAND:                  # the dense copy sits at the head of the workspace
         eb = 1 if w.desc.dtype == nm.NM_I8 else 2
         plan.workspace_bytes += -(-(w.desc.O * (-(-(w.desc.K * eb) // 16) * 16)) // 256) * 256
@@ -42,6 +46,8 @@ def make_plan(T, w, od, **over):
 
 def gpu_spmm(X: np.ndarray, W: np.ndarray, n: int, m: int, od: int | None = None, images=nm.NM_IMG_AUTO, **plan_over):
     """Returns (Y numpy, plan dict, packed weight).  Raises on a device-side timeout."""
+    if plan_over.get("path") == nm.NM_PATH_UMMA_REMAP48 and images == nm.NM_IMG_AUTO:
+        images = nm.NM_IMG_AUTO | nm.NM_IMG_REMAP48         # only built on request
     if plan_over.get("path") == nm.NM_PATH_UMMA_SP24 and images == nm.NM_IMG_AUTO:
         images = nm.NM_IMG_AUTO | nm.NM_IMG_HW24            # short rows get only the dense image by default
     w = nm.nm_compress(W, n, m, images=images)

@@ -40,22 +40,25 @@ def test_canonical_bytes_equal_oracle(n, m, dtype):
     assert np.array_equal(canon, orc.compress(W, n, m))
 
 
-def _decode_hw24(pw, dtype):
+def _decode_hw24(pw, dtype, remap=False):
     """Test-side reader of the hardware 2:4 image: rebuilds W~ from compressed values and
-    the 4-bit-per-chunk metadata (two ascending 2-bit positions, low slot first)."""
+    the 4-bit-per-chunk metadata (two ascending 2-bit positions, low slot first).  remap=True reads
+    the 2:4 image of the K-remapped weight instead (same format, longer K)."""
     d = pw.desc
-    O, K = d.O, d.K
+    O, K = d.O, (d.remap_k if remap else d.K)
+    off_v, off_m, row_bytes, kblocks = ((d.off_remap_values, d.off_remap_meta, d.remap_row_bytes, d.remap_meta_kblocks) if remap else
+                                        (d.off_hw24_values, d.off_hw24_meta, d.hw24_row_bytes, d.hw24_meta_kblocks))
     eb = 1 if dtype == "i8" else 2
     chunks = (K + 3) // 4
-    vals = pw.buf[d.off_hw24_values:d.off_hw24_values + O * d.hw24_row_bytes].reshape(O, d.hw24_row_bytes)
+    vals = pw.buf[off_v:off_v + O * row_bytes].reshape(O, row_bytes)
     vals = vals.view(np.int8 if dtype == "i8" else np.float16)
-    meta = pw.buf[d.off_hw24_meta:]
+    meta = pw.buf[off_m:]
     W = np.zeros((O, chunks * 4), dtype=vals.dtype)
     for o in range(O):
         ot, r = divmod(o, 128)
         for c in range(chunks):
             kb, cc = divmod(c, 32)
-            blk = (ot * d.hw24_meta_kblocks + kb) * 2048
+            blk = (ot * kblocks + kb) * 2048
             if eb == 1:
                 byte, shift = r * 16 + cc // 2, (cc & 1) * 4
             else:
@@ -78,6 +81,44 @@ def test_hw24_image_roundtrip(n, m, dtype):
     pw = nm.nm_compress_host(W, n, m)
     assert pw.desc.images & nm.NM_IMG_HW24 and not pw.desc.images & nm.NM_IMG_DENSE
     assert np.array_equal(_decode_hw24(pw, dtype), W)
+
+
+@pytest.mark.parametrize("n,m", [(4, 8), (3, 8), (2, 8)])
+@pytest.mark.parametrize("dtype", ["i8", "f16"])
+def test_remap48_image_folds_back_to_the_weight(n, m, dtype):
+    """Three-chunk K remap: the remapped weight is 2:4-clean (the 2:4 packer accepted it), holds the
+    moved elements in the third chunks, and folding those back onto k + {0,1,4,5} restores W."""
+    O, K = 150, 264 if dtype == "i8" else 136          # K is not a multiple of the sparse K step: the main range is padded
+    W = (inputs.w_i8 if dtype == "i8" else inputs.w_f16)(O, K, n, m, "remap", at_most=True)
+    if n == 4:                                          # worst cases: all four nonzeros of a group in one 4-chunk
+        W[0, :] = 0
+        W[0, 0:4] = 3
+        W[1, :] = 0
+        W[1, 12:16] = -5
+    pw = nm.nm_compress_host(W, n, m, images=nm.NM_IMG_AUTO | nm.NM_IMG_REMAP48)
+    d = pw.desc
+    assert d.images & nm.NM_IMG_REMAP48
+    eb = 1 if dtype == "i8" else 2
+    assert d.remap_k_main == -(-K * eb // 256) * 256 // eb and d.remap_k == d.remap_k_main + K // 2
+    Wr = _decode_hw24(pw, dtype, remap=True)
+    assert (np.count_nonzero(Wr.reshape(O, -1, 4), axis=2) <= 2).all()
+    assert not Wr[:, K:d.remap_k_main].any()
+    back = Wr[:, :K].copy()
+    third = Wr[:, d.remap_k_main:].reshape(O, K // 8, 4)
+    for j, pos in enumerate((0, 1, 4, 5)):
+        cols = np.arange(K // 8) * 8 + pos
+        assert not (back[:, cols] != 0)[third[:, :, j] != 0].any(), "a moved element must leave its original place"
+        back[:, cols] += third[:, :, j]
+    assert np.array_equal(back, W)
+    if n == 4:
+        assert np.count_nonzero(third) > 0
+    # a weight with more than 4 nonzeros in a group of 8 cannot be remapped; dense weights need no image
+    W58 = inputs.w_i8(8, 64, 5, 8, "remap58")
+    with pytest.raises(nm.NMError) as e:
+        nm.nm_compress_host(W58, 5, 8, images=nm.NM_IMG_AUTO | nm.NM_IMG_REMAP48)
+    assert e.value.status == nm.NM_ERR_UNSUPPORTED
+    # never built unless asked for
+    assert not nm.nm_compress_host(W, n, m).desc.images & nm.NM_IMG_REMAP48
 
 
 def test_image_selection():
