@@ -72,7 +72,10 @@ enum {
   NM_PATH_UMMA_DENSE = 1, /* TMA -> smem -> dense tcgen05.mma, accumulators in TMEM        */
   NM_PATH_UMMA_SP24 = 2,  /* TMA -> smem -> tcgen05.mma.sp (2:4 hardware sparsity)         */
   NM_PATH_UMMA_DECODE = 3,/* canonical image -> decode warps build the zero-filled micro-dense
-                             tile in smem -> dense tcgen05.mma; any n:m, no extra image   */
+                             tile in smem -> dense tcgen05.mma; any n:m, no extra image.  A
+                             correctness fallback for callers with neither a pre-arranged image nor
+                             scratch: every W tile is decoded again for every token tile that meets
+                             it, measured 2-17x the time of NM_PATH_UMMA_EXPAND / a dense image   */
   NM_PATH_UMMA_EXPAND = 4,/* canonical image -> one small kernel writes the zero-filled dense rows
                              once into the head of the workspace (O x round_up(K*eb,16) bytes,
                              counted in nm_plan.workspace_bytes; it stays in L2) -> the dense
