@@ -150,7 +150,7 @@ int main() {
   }
   // ---- part 2
   unsigned long long* out; cudaMalloc(&out, 16 * 148);
-  for (size_t mb : {32, 1024}) {
+  for (size_t mb : {32, 64, 96, 1024}) {
     uint8_t* buf; cudaMalloc(&buf, mb << 20); cudaMemset(buf, 1, mb << 20);
     for (int box_rows : {64, 128, 256}) for (int boxes : {1, 2}) { run_ring<2>(enc, buf, mb, out, box_rows, boxes, sms); run_ring<4>(enc, buf, mb, out, box_rows, boxes, sms); }
     cudaFree(buf);

@@ -39,6 +39,7 @@ def main():
     ap.add_argument("--tile-t", type=int, default=0, help="override the token tile of every plan (0: the planner's)")
     ap.add_argument("--split-k", type=int, default=0, help="override split-K of every plan that splits (0: the planner's)")
     ap.add_argument("--issuers", type=int, default=0)
+    ap.add_argument("--cta-group", type=int, default=0)
     ap.add_argument("--out", default=None)
     args = ap.parse_args()
 
@@ -69,6 +70,8 @@ def main():
             plan.stages = args.stages
         if args.issuers:
             plan.issuers = args.issuers
+        if args.cta_group:
+            plan.cta_group = args.cta_group
         if args.tile_t or args.split_k:
             plan.tile_t = args.tile_t or plan.tile_t
             if args.split_k:

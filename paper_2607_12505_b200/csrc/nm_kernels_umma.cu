@@ -34,6 +34,7 @@
 // status word, raises a CTA-wide abort flag that every role polls, frees its tensor memory
 // and returns.
 #include <atomic>
+#include <cstdlib>
 
 #include "nm_umma_common.cuh"
 
@@ -82,6 +83,7 @@ struct UmmaParams {
   uint32_t spin_limit;      // polls after which a bounded wait gives up
   int diag_stall;           // diagnostic (NM_PLAN_DIAG_STALL): CTA 0 arms its first K step for 16 bytes that never come
   unsigned long long* trace;   // phase stamps (trace builds only; nullptr otherwise)
+  int dbg;                     // trace builds only: 1 = no MMAs are issued, 2 = no output is stored, 3 = both (timing experiments)
   uint32_t* status;
   // decode path: the canonical image (values + bit-packed positions)
   const uint8_t* canon_vals; const uint8_t* canon_idx;
@@ -543,7 +545,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         if (use >= 1u) {     // the epilogue must have drained this accumulator buffer
           NM_WAIT_TIMED(cyc_tempty, ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, wctx, 4));
-          ok = __all_sync(0xffffffffu, ok);
+          ok = __all_sync(0xffffffffu, ok);        // every lane polls; also re-converges the warp after the poll loop
           if (!ok) break;
           tc_fence_after();
         }
@@ -558,7 +560,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             continue;
           }
           NM_WAIT_TIMED(cyc_full, ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2));
-          ok = __all_sync(0xffffffffu, ok);        // also re-converges the warp after the poll loop
+          ok = __all_sync(0xffffffffu, ok);        // every lane polls; also re-converges the warp after the poll loop
           if (!ok) break;
           tc_fence_after();
           if (n == 0 && i == (int)which && lane == 0 && which == 0u) NM_STAMP(p.trace, 3);
@@ -568,6 +570,9 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t sb = res_x ? slot : st;
           // metadata columns follow the copy of the metadata they hold: ring stage or K step
           const uint32_t meta_cols = tmem_meta + (res_w ? (uint32_t)ks : s) * 8u;
+#ifdef NM_TRACE
+          if (p.dbg & 1) { tc_commit(bar_empty + 8u * s); if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; st = ring_base; } else { st += sbytes; } continue; }
+#endif
           if (SP) {
             const uint32_t sm = sa + 16384u;
             tc_cp_128x128b(meta_cols, desc_meta(sm));
@@ -646,6 +651,9 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int cc = (h ^ (n & 1)) * 32; cc < p.tile_t; cc += 64) {
         const int t = c.t0 + cc;
         if (t >= p.T) break;
+#ifdef NM_TRACE
+        if (p.dbg & 2) continue;
+#endif
         uint32_t r[32];
         if (CLU) {
           // Split-K met on chip (Section 4.3: partial sums are merged only in the final stage).
@@ -1030,6 +1038,9 @@ nm_status launch_umma(const SpmmArgs& a) {
   p.diag_stall = (pl.reserved & NM_PLAN_DIAG_STALL) ? 1 : 0;
   p.spin_limit = p.diag_stall ? (1u << 14) : kSpinLimit;
   p.trace = trace_buffer();
+#ifdef NM_TRACE
+  { const char* e = getenv("NM_DBG"); p.dbg = e ? atoi(e) : 0; }
+#endif
   if (dec) {
     CanonGeom g;
     nm_status gs = canon_geom(w->O, w->K, w->n, w->m, w->dtype, &g);

@@ -16,6 +16,7 @@
 // single-CTA kernel.  All waits are bounded polls; the two CTAs meet at a cluster barrier
 // before tensor memory is freed, so neither can exit while the other still targets it.
 #include <atomic>
+#include <cstdlib>
 
 #include "nm_umma_common.cuh"
 
@@ -43,6 +44,7 @@ struct PairParams {
   uint32_t tmem_cols;
   uint32_t spin_limit;      // polls after which a bounded wait gives up
   unsigned long long* trace;   // phase stamps (trace builds only; nullptr otherwise)
+  int dbg;                     // trace builds only: 1 = no MMAs are issued, 2 = no output is stored, 3 = both (timing experiments)
   uint32_t* status;
 };
 
@@ -272,7 +274,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t buf = (uint32_t)n % (uint32_t)p.acc_bufs, use = (uint32_t)n / (uint32_t)p.acc_bufs;
         if (use >= 1u) {       // both CTAs' epilogues must have drained this accumulator buffer
           NM_WAIT_TIMED(cyc_tempty, ok = mbar_wait(bar_tempty + 8u * buf, (use - 1u) & 1u, wctx, 4));
-          ok = __all_sync(0xffffffffu, ok);
+          ok = __all_sync(0xffffffffu, ok);        // every lane polls; also re-converges the warp after the poll loop
           if (!ok) break;
           tc_fence_after();
         }
@@ -283,13 +285,16 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (o_idx >= p.tiles_o2) { o_idx -= p.tiles_o2; ++t_idx; }
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
           NM_WAIT_TIMED(cyc_full, ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2));
-          ok = __all_sync(0xffffffffu, ok);        // also re-converges the warp after the poll loop
+          ok = __all_sync(0xffffffffu, ok);        // every lane polls; also re-converges the warp after the poll loop
           if (!ok) break;
           tc_fence_after();
           if (n == 0 && ks == 0 && lane == 0) NM_STAMP(p.trace, 3);
           const uint32_t sm = sa + 16384u;
           const uint32_t sb = sm + meta_bytes2<DT, SP>();
           const uint32_t meta_cols = tmem_meta + s * 8u;
+#ifdef NM_TRACE
+          if (p.dbg & 1) { tc_commit_pair(bar_empty + 8u * s); if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; sa = smem_base; } else { sa += sbytes; } continue; }
+#endif
           if (SP) {
             tc_cp_128x128b_pair(meta_cols, desc_meta(sm));
             if (DT == NM_I8) tc_cp_128x128b_pair(meta_cols + 4u, desc_meta(sm + 2048u));
@@ -351,6 +356,9 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int t = t0 + cc;
         if (t >= p.T) break;
         uint32_t r[32];
+#ifdef NM_TRACE
+        if (p.dbg & 2) continue;
+#endif
         if (lane == 0) tma_store_wait_read();
         __syncwarp();
         tc_ld_32x32(lane_addr + (uint32_t)cc, r);
@@ -502,6 +510,9 @@ nm_status launch_umma_pair(const SpmmArgs& a, bool* handled) {
   p.status = a.status;
   p.spin_limit = kSpinLimit;
   p.trace = trace_buffer();
+#ifdef NM_TRACE
+  { const char* e = getenv("NM_DBG"); p.dbg = e ? atoi(e) : 0; }
+#endif
   p.w_fresh = a.w_fresh ? 1 : 0;
   p.tiles_o2 = ceil_div(w->O, 256);
   const int64_t items = (int64_t)p.tiles_o2 * ceil_div(a.T, pl.tile_t);
