@@ -11,6 +11,10 @@ just before tensor memory is freed.  The launches are replayed as one CUDA graph
 launches, as in a model); the table gives, per layer of the last replay, the earliest / median /
 latest CTA for every phase relative to the release of the grid-dependency wait, and the gap
 between the end of one layer and the release of the next one's wait.
+
+Timing experiments of the trace build (environment variable NM_DBG, read at launch): 1 = the issuing
+warp issues no MMAs (stages are recycled at once), 2 = the epilogue stores nothing, 3 = both, i.e. only
+the operand loads run.  Results are wrong by construction; only the times mean something.
 """
 from __future__ import annotations
 
