@@ -81,6 +81,10 @@ nm_status plan_shape(int T, int O, int K, int n, int m, int dt, int od, uint32_t
     for (int cand = 32; cand <= 256; cand += 32) {
       if (cand > t_cap) break;
       if (cand < 64 && t_cap >= 64 && T > 256) continue;  // 32-token tiles only for small token counts
+      // Dense-MMA CTA pairs: two 256-token accumulators fill tensor memory exactly (no metadata columns)
+      // and a 256-token tile moves the fewest operand bytes per MMA; on every shape swept the pair kernel
+      // was fastest there (3-14 % ahead of the 160-224 tokens the cost terms below would pick).
+      if (cg == 2 && !sp && T >= 512 && cand != 256) continue;
       // the last token tile is multiplied over its occupied 32-token chunks only
       const int rag_tokens = T % cand, rag_n = (rag_tokens + 31) / 32 * 32;
       for (int s = 1; s <= kMaxSplitK; s *= 2) {
