@@ -14,7 +14,9 @@ between the end of one layer and the release of the next one's wait.
 
 Timing experiments of the trace build (environment variable NM_DBG, read at launch): 1 = the issuing
 warp issues no MMAs (stages are recycled at once), 2 = the epilogue stores nothing, 3 = both, i.e. only
-the operand loads run.  Results are wrong by construction; only the times mean something.
+the operand loads run; 4 (CTA-pair kernel only) = the ring is loaded once and the K loops run over it
+without further loads, so 6 = the MMAs alone.  Results are wrong by construction; only the times mean
+something.
 """
 from __future__ import annotations
 

@@ -44,7 +44,7 @@ struct PairParams {
   uint32_t tmem_cols;
   uint32_t spin_limit;      // polls after which a bounded wait gives up
   unsigned long long* trace;   // phase stamps (trace builds only; nullptr otherwise)
-  int dbg;                     // trace builds only: 1 = no MMAs are issued, 2 = no output is stored, 3 = both (timing experiments)
+  int dbg;                     // trace builds only, bits: 1 = no MMAs are issued, 2 = no output is stored, 4 = the ring is loaded once and reused (timing experiments; wrong results)
   uint32_t* status;
 };
 
@@ -189,6 +189,9 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int t0 = tile0 + (int)rank * (int)half_rows;
         if (p.T - tile0 < p.tile_t) t0 = tile0 + (int)rank * (((p.T - tile0 + 31) & ~31) >> 1);
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
+#ifdef NM_TRACE
+          if ((p.dbg & 4) && armed >= (uint32_t)p.stages) { n = my_count; break; }   // the ring is filled once and reused
+#endif
           if (wrapped) {
             NM_WAIT_TIMED(cyc_empty, ok = mbar_wait(bar_empty + 8u * s, ph ^ 1u, wctx, 1));
             if (!ok) break;
@@ -284,6 +287,9 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         t_idx += step_t; o_idx += step_o;
         if (o_idx >= p.tiles_o2) { o_idx -= p.tiles_o2; ++t_idx; }
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
+#ifdef NM_TRACE
+          if (!((p.dbg & 4) && (n > 0 || ks >= p.stages)))      // 4 = no loads after the first ring-full: the MMAs run alone
+#endif
           NM_WAIT_TIMED(cyc_full, ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2));
           ok = __all_sync(0xffffffffu, ok);        // every lane polls; also re-converges the warp after the poll loop
           if (!ok) break;
