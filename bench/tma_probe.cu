@@ -98,6 +98,61 @@ __global__ void __launch_bounds__(128, 1) ring_kernel(const __grid_constant__ CU
   }
 }
 
+// part 3: the operand pattern of a GEMM (T x K activations, O x K weights, 128-byte K slices, out-feature tiles varying
+// fastest over the CTAs, so weight boxes are shared by ~1/6 of the CTAs and activation boxes by 6) in a ring whose
+// producer thread waits for a consumer warp (all lanes poll the full barrier, lane 0 releases the stage), as the
+// GEMM kernels do.  `extra` dependent integer instructions per stage show what the producer's own instruction time costs.
+template <int S>
+__global__ void __launch_bounds__(128, 1) gemm_ring_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                                                           unsigned long long* outg, int items, int tiles_o, int ksteps, int tile_t, int extra, int cextra) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t bbytes = (uint32_t)tile_t * 128u, abytes = 16384u, sb = bbytes + abytes;
+  const uint32_t full = base + S * sb, empty = full + 8 * S;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 2 * S; ++s) mbar_init(full + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long t0, t1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    bool ok = true, wrapped = false;
+    uint32_t s = 0, ph = 0, v = 1; long steps = 0;
+    for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+      const int o0 = (item % tiles_o) * 128, t0r = (item / tiles_o) * tile_t;
+      for (int ks = 0; ks < ksteps; ++ks) {
+        if (wrapped) { ok = mbar_wait(empty + 8 * s, ph ^ 1u); if (!ok) break; }
+        const uint32_t st = base + s * sb;
+        mbar_expect_tx(full + 8 * s, sb);
+        tma_load_2d(st, &tmB, full + 8 * s, ks * 128, t0r);
+        tma_load_2d(st + bbytes, &tmA, full + 8 * s, ks * 128, o0);
+        for (int q = 0; q < extra; ++q) asm volatile("mad.lo.u32 %0, %0, %0, %1;" : "+r"(v) : "r"(q));
+        ++steps;
+        if (++s == S) { s = 0; ph ^= 1u; wrapped = true; }
+      }
+    }
+    for (int d = 0; d < S && ok; ++d)      // let the last loads land before the CTA gives up its shared memory
+      if (steps > d) { const long g = steps - 1 - d; ok = mbar_wait(full + 8 * (uint32_t)(g % S), (uint32_t)((g / S) & 1)); }
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+    outg[blockIdx.x * 3] = t0; outg[blockIdx.x * 3 + 1] = (ok && v != 0x7fffffffu) ? t1 : 0; outg[blockIdx.x * 3 + 2] = (unsigned long long)steps;
+  } else if (threadIdx.x >= 32 && threadIdx.x < 64) {
+    const int lane = threadIdx.x & 31;
+    uint32_t s = 0, ph = 0, v = 1; bool ok = true;
+    for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+      for (int ks = 0; ks < ksteps; ++ks) {
+        ok = mbar_wait(full + 8 * s, ph);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        for (int q = 0; q < cextra; ++q) asm volatile("mad.lo.u32 %0, %0, %0, %1;" : "+r"(v) : "r"(q));      // stands for the consumer's own work
+        if (lane == 0 && v != 0x7fffffffu) mbar_arrive(empty + 8 * s);
+        __syncwarp();
+        if (++s == S) { s = 0; ph ^= 1u; }
+      }
+    }
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
@@ -128,6 +183,27 @@ static void run_ring(EncodeTiledFn enc, uint8_t* buf, size_t mb, unsigned long l
   }
 }
 
+static bool make_map_rows(EncodeTiledFn enc, CUtensorMap* tm, void* buf, uint64_t row_bytes, uint64_t rows, uint32_t box_rows) {
+  return make_map(enc, tm, buf, row_bytes, rows, box_rows);
+}
+template <int S>
+static void run_gemm_ring(EncodeTiledFn enc, uint8_t* W, uint8_t* X, unsigned long long* out, int T, int O, int K, int tile_t, int extra, int grid, int cextra = 0) {
+  CUtensorMap tmA, tmB;
+  if (!make_map_rows(enc, &tmA, W, K, O, 128) || !make_map_rows(enc, &tmB, X, K, T, tile_t)) { printf("tensor map failed\n"); return; }
+  const size_t smem = 1024 + (size_t)S * (tile_t * 128 + 16384) + 16 * S + 64;
+  if (smem > 227 * 1024) return;
+  cudaFuncSetAttribute(gemm_ring_kernel<S>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const int tiles_o = O / 128, tiles_t = (T + tile_t - 1) / tile_t, items = tiles_o * tiles_t, ksteps = K / 128;
+  for (int rep = 0; rep < 3; ++rep) { gemm_ring_kernel<S><<<grid, 128, smem>>>(tmA, tmB, out, items, tiles_o, ksteps, tile_t, extra, cextra); cudaDeviceSynchronize(); }
+  std::vector<unsigned long long> h(grid * 3);
+  cudaMemcpy(h.data(), out, grid * 24, cudaMemcpyDeviceToHost);
+  unsigned long long t0 = ~0ull, t1 = 0, maxsteps = 0, tot = 0; bool ok = true;
+  for (int i = 0; i < grid; ++i) { if (!h[3 * i + 1]) ok = false; if (h[3 * i] < t0) t0 = h[3 * i]; if (h[3 * i + 1] > t1) t1 = h[3 * i + 1]; if (h[3 * i + 2] > maxsteps) maxsteps = h[3 * i + 2]; tot += h[3 * i + 2]; }
+  const double bytes = (double)tot * (tile_t * 128.0 + 16384.0);
+  printf("gemm ring: T %d O %d K %d, token tile %3d, %d stages, %3d / %3d extra producer / consumer instructions per stage: %s span %.2f us, %.3f us per stage of the busiest CTA, %.1f TB/s into shared memory  (%s)\n",
+         T, O, K, tile_t, S, extra, cextra, ok ? "ok" : "WAIT EXPIRED", (t1 - t0) / 1e3, (t1 - t0) / 1e3 / (double)maxsteps, bytes / (double)(t1 - t0) / 1e3, cudaGetErrorString(cudaGetLastError()));
+}
+
 int main() {
   void* sym = nullptr; cudaDriverEntryPointQueryResult q;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym) { printf("no cuTensorMapEncodeTiled\n"); return 1; }
@@ -154,6 +230,22 @@ int main() {
     uint8_t* buf; cudaMalloc(&buf, mb << 20); cudaMemset(buf, 1, mb << 20);
     for (int box_rows : {64, 128, 256}) for (int boxes : {1, 2}) { run_ring<2>(enc, buf, mb, out, box_rows, boxes, sms); run_ring<4>(enc, buf, mb, out, box_rows, boxes, sms); }
     cudaFree(buf);
+  }
+  // ---- part 3: DeiT-B fc2 (25216 tokens, K = 3072 -> 768 out-features), one CTA per SM
+  {
+    const int T = 25216, O = 768, K = 3072;
+    uint8_t *W, *X; unsigned long long* out3;
+    cudaMalloc(&W, (size_t)O * K); cudaMalloc(&X, (size_t)T * K); cudaMalloc(&out3, 24 * 148);
+    cudaMemset(W, 1, (size_t)O * K); cudaMemset(X, 1, (size_t)T * K);
+    for (int extra : {0, 16, 32, 64, 128}) {
+      run_gemm_ring<4>(enc, W, X, out3, T, O, K, 256, extra, sms);
+      run_gemm_ring<4>(enc, W, X, out3, T, O, K, 128, extra, sms);
+    }
+    for (int cextra : {32, 64, 128}) run_gemm_ring<4>(enc, W, X, out3, T, O, K, 256, 0, sms, cextra);
+    run_gemm_ring<4>(enc, W, X, out3, T, O, K, 256, 32, sms, 64);
+    run_gemm_ring<2>(enc, W, X, out3, T, O, K, 128, 0, sms);
+    run_gemm_ring<6>(enc, W, X, out3, T, O, K, 128, 0, sms);
+    cudaFree(W); cudaFree(X); cudaFree(out3);
   }
   return 0;
 }
