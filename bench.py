@@ -20,7 +20,8 @@ peak measured in the same run (sparse = twice that) and against the nominal 4.5 
 computes are compared bit for bit with what the timed kernels left in Y (`verified`).  Further legs,
 each a replayed CUDA graph timed with CUDA events: the DeiT-Small stack (`cfg1_step`), the same
 DeiT-Base stack in FP16 (`cfg2_fp16`), the 72 linear layers of ViT-Large at batch 1 (`vit_l_b1_stack`),
-one ViT-Large batch-256 fc2 GEMM (`vit_l_b256_fc2`), dense cuBLAS on the same buffers (`cublas_dense`).
+one ViT-Large batch-256 fc2 GEMM with INT32 and with fused-requantised INT8 results (`vit_l_b256_fc2`,
+`vit_l_b256_fc2_int8_out`), dense cuBLAS on the same buffers (`cublas_dense`).
 """
 from __future__ import annotations
 
@@ -635,6 +636,29 @@ def extra_legs(torch, nm, dev, stream, hbm_peak, main_workload):
                              "frac_of_sparse_peak_measured": t_ops / (2 * int8_peak), "frac_of_sparse_peak_nominal_9000": t_ops / 9000.0,
                              "int8_dense_peak_tops_measured": round(int8_peak, 1), "gbs": algorithmic_bytes(spec) / ms / 1e6,
                              "frac_of_hbm": algorithmic_bytes(spec) / ms / 1e6 / hbm_peak, "status_ok": all(v == 0 for v in st.status_words())}
+
+    # --- the same GEMM through the fused requantising epilogue (INT8 results: a quarter of the write-back), per-channel scale 1e-4
+    scale = torch.full((spec["O"],), 1e-4, dtype=torch.float32, device=dev)
+    Y8 = [torch.empty((spec["T"], spec["O"]), dtype=torch.int8, device=dev) for _ in st.layers]
+    plans8 = [nm.nm_plan_create(spec["T"], Lq["w"], nm.NM_OUT_I8, dev.index) for Lq in st.layers]
+    ws8 = [torch.empty(max(int(p.workspace_bytes), 256), dtype=torch.uint8, device=dev) for p in plans8]
+    st8 = torch.zeros(len(st.layers), dtype=torch.int32, device=dev)
+
+    def q_step():
+        for i, (Lq, y, pl, w8) in enumerate(zip(st.layers, Y8, plans8, ws8)):
+            nm.nm_spmm(Lq["Xd"], Lq["w"], plan=pl, out=y, out_dtype=nm.NM_OUT_I8, workspace=w8, status=st8[i:i + 1], stream=stream, scale=scale)
+    ms8 = time_graph(torch, stream, graph_of(torch, stream, q_step, 5), 3) / 10
+    # every element against the INT32 result of the run above, requantised with the same single IEEE operations
+    ref8 = torch.clamp(torch.round(L["Yd"].to(torch.float32) * scale[None, :]), -128, 127).to(torch.int8)
+    same = bool(torch.equal(ref8, Y8[0]))
+    t_ops8 = dense_ops(spec) / ms8 / 1e9
+    out["vit_l_b256_fc2_int8_out"] = {"us": ms8 * 1e3, "dense_tops": t_ops8, "speedup_vs_cublas_dense_int32_out": cb / ms8,
+                                      "frac_of_sparse_peak_measured": t_ops8 / (2 * int8_peak),
+                                      "frac_of_sparse_peak_nominal_9000": t_ops8 / 9000.0,
+                                      "plan": {k: v for k, v in plans8[0].as_dict().items() if k in ("path", "tile_t", "cta_group", "split_k", "issuers")},
+                                      "equals_requantised_int32_result": same,
+                                      "status_ok": all(int(v) == 0 for v in st8.cpu().tolist()),
+                                      "what": "nm_spmm_ex with a per-channel scale: INT8 in, INT8 out, the paper's INT8 pipeline between two linear layers"}
     return out
 
 
