@@ -19,7 +19,7 @@ peak measured in the same run (sparse = twice that) and against the nominal 4.5 
 `cpu_baseline` times the CPU oracle on a bounded row sample of the same workload, and the rows it
 computes are compared bit for bit with what the timed kernels left in Y (`verified`).  Further legs,
 each a replayed CUDA graph timed with CUDA events: the DeiT-Small stack (`cfg1_step`), the same
-DeiT-Base stack in FP16 (`cfg2_fp16`), the 72 linear layers of ViT-Large at batch 1 (`vit_l_b1_stack`),
+DeiT-Base stack in FP16 (`cfg2_fp16`) and with fused-requantised INT8 results (`cfg2_int8_out`), the 72 linear layers of ViT-Large at batch 1 (`vit_l_b1_stack`),
 one ViT-Large batch-256 fc2 GEMM with INT32 and with fused-requantised INT8 results (`vit_l_b256_fc2`,
 `vit_l_b256_fc2_int8_out`), dense cuBLAS on the same buffers (`cublas_dense`).
 """
@@ -144,7 +144,7 @@ def run_reference(args, wl):
 class Stack:
     """A list of GEMMs on one device, every GEMM with its own X, Y, packed W, scratch and status word."""
 
-    def __init__(self, torch, nm, specs, dev, key, rank=0, od=None, host_x=False, device_x=False):
+    def __init__(self, torch, nm, specs, dev, key, rank=0, od=None, host_x=False, device_x=False, scale=None):
         self.torch, self.nm, self.dev = torch, nm, dev
         self.layers = []
         for s in specs:
@@ -164,7 +164,12 @@ class Stack:
             plan = nm.nm_plan_create(s["T"], w, odt, dev.index)
             Yd = torch.empty((s["T"], s["O"]), dtype=nm._out_torch_dtype(odt), device=dev)
             ws = torch.empty(max(int(plan.workspace_bytes), 256), dtype=torch.uint8, device=dev)
-            self.layers.append(dict(spec=s, w=w, plan=plan, Xh=Xh, Xd=Xd, Yd=Yd, ws=ws, W=W, X=X, od=odt))
+            epi = sc = None
+            if scale is not None:      # fused requantising epilogue: one fp32 scale per out-feature
+                import ctypes
+                sc = torch.full((s["O"],), float(scale), dtype=torch.float32, device=dev)
+                epi = nm.NMEpilogue(sc.data_ptr(), None, 0, 0)
+            self.layers.append(dict(spec=s, w=w, plan=plan, Xh=Xh, Xd=Xd, Yd=Yd, ws=ws, W=W, X=X, od=odt, epi=epi, scale=sc))
         self.status = torch.zeros(len(self.layers), dtype=torch.int32, device=dev)
 
     def kernel_of(self, L):
@@ -177,9 +182,15 @@ class Stack:
         for i, L in enumerate(self.layers):
             if only is not None and self.kernel_of(L) != only:
                 continue
-            st = nm.nm_spmm_raw(L["Xd"].data_ptr(), L["spec"]["K"], L["spec"]["T"], L["w"], L["plan"], L["Yd"].data_ptr(),
-                                L["spec"]["O"], L["od"], L["ws"].data_ptr(), L["ws"].numel(),
-                                self.status.data_ptr() + 4 * i, sptr)
+            if L["epi"] is not None:
+                import ctypes
+                st = nm.lib().nm_spmm_ex(L["Xd"].data_ptr(), L["spec"]["K"], L["spec"]["T"], ctypes.byref(L["w"].desc), ctypes.byref(L["plan"]),
+                                         L["Yd"].data_ptr(), L["spec"]["O"], L["od"], ctypes.byref(L["epi"]), L["ws"].data_ptr(), L["ws"].numel(),
+                                         self.status.data_ptr() + 4 * i, ctypes.c_void_p(sptr))
+            else:
+                st = nm.nm_spmm_raw(L["Xd"].data_ptr(), L["spec"]["K"], L["spec"]["T"], L["w"], L["plan"], L["Yd"].data_ptr(),
+                                    L["spec"]["O"], L["od"], L["ws"].data_ptr(), L["ws"].numel(),
+                                    self.status.data_ptr() + 4 * i, sptr)
             if st != nm.NM_OK:
                 raise RuntimeError(f"nm_spmm failed: {nm.lib().nm_status_string(st).decode()}")
 
@@ -591,6 +602,23 @@ def extra_legs(torch, nm, dev, stream, hbm_peak, main_workload):
                             "gbs": by / ms / 1e6, "frac_of_hbm": by / ms / 1e6 / hbm_peak, "status_ok": ok}
         del st
         torch.cuda.empty_cache()
+
+    # --- the headline stack with INT8 results (fused requantising epilogue, per-channel scale 1e-4): the INT8 pipeline
+    #     between linear layers; the first four GEMMs are checked, every element, against a dense library GEMM requantised by torch
+    specs = inputs.cfg2_layers("i8")
+    st = Stack(torch, nm, specs, dev, "bench_q8", device_x=True, od=nm.NM_OUT_I8, scale=1e-4)
+    ms = time_graph(torch, stream, st.graph(stream), 10)
+    same = True
+    for Lq in st.layers[:4]:
+        acc = torch._int_mm(Lq["Xd"], torch.from_numpy(Lq["W"]).to(dev).t())          # comparator only
+        ref = torch.clamp(torch.round(acc.to(torch.float32) * Lq["scale"][None, :]), -128, 127).to(torch.int8)
+        same = same and bool(torch.equal(ref, Lq["Yd"]))
+        del acc, ref
+    out["cfg2_int8_out"] = {"workload": "deit_base_12block_linear_stack_int8_in_int8_out_b128", "ms_per_step": ms,
+                            "dense_tops": sum(dense_ops(s) for s in specs) / ms / 1e9,
+                            "first_gemms_equal_requantised_dense_library_gemm": same, "status_ok": all(v == 0 for v in st.status_words())}
+    del st
+    torch.cuda.empty_cache()
 
     # --- the DeiT-Base stack in FP16 (fp32 accumulation, fp16 out), against torch.matmul on the same buffers
     specs = inputs.cfg2_layers("f16")
