@@ -398,10 +398,11 @@ def main():
             def cublas_step():
                 for i, (L, Wd) in enumerate(zip(layers, Wds)):
                     outs[i] = torch._int_mm(L["Xd"], Wd.t())      # comparator only; never on the product path
-            cublas_ms = graph_us(cublas_step, 5) / 1e3
+            # the same number of back-to-back steps as the headline, so that both see the same clocks (a long run is power-limited)
+            cublas_ms = time_graph(torch, stream, graph_of(torch, stream, cublas_step, 1), max(args.steps, 3))
             del outs
             cublas = {"ms_per_step": cublas_ms, "launch": "cuda_graph_replay", "library": "torch._int_mm (cuBLASLt heuristic)",
-                      "speedup_vs_cublas_dense": cublas_ms / ms_per_step}
+                      "timed_over_steps": max(args.steps, 3), "speedup_vs_cublas_dense": cublas_ms / ms_per_step}
             seen = {}
             for L, Wd in zip(layers, Wds):
                 s = L["spec"]
