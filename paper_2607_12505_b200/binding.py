@@ -111,6 +111,8 @@ def lib() -> ctypes.CDLL:
         return _lib
     if os.environ.get("NM_B200_TRACE") == "1":      # the trace build (phase stamps), for bench.trace_phases only
         path = _build.build(trace=True)
+    elif os.environ.get("NM_B200_TRACE") == "2":    # the NM_DBG timing experiments without stamp code (harness only)
+        path = _build.build(dbg_modes=True)
     else:
         path = _build.LIB
         if _build.is_stale():

@@ -38,18 +38,22 @@ def is_stale(lib: str = LIB) -> bool:
 
 
 TRACE_LIB = os.path.join(_HERE, "libnm_b200_trace.so")
+DBG_LIB = os.path.join(_HERE, "libnm_b200_dbg.so")
 
 
-def build(force: bool = False, verbose: bool = False, trace: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, trace: bool = False, dbg_modes: bool = False) -> str:
     """trace=True builds a second library with -DNM_TRACE (phase stamps in the tcgen05 kernels, used
-    by `python -m bench.trace_phases`); the product library never contains the stamps."""
-    lib = TRACE_LIB if trace else LIB
+    by `python -m bench.trace_phases`); dbg_modes=True a third one with -DNM_DBG_MODES (the NM_DBG timing
+    experiments without any stamp code).  The product library contains neither."""
+    lib = TRACE_LIB if trace else (DBG_LIB if dbg_modes else LIB)
     if not force and not is_stale(lib):
         return lib
     tmp = lib + f".tmp{os.getpid()}"
     cmd = [_nvcc(), *NVCC_FLAGS, "-I", os.path.join(_ROOT, "include"), "-I", CSRC]
     if trace:
         cmd += ["-DNM_TRACE"]
+    elif dbg_modes:
+        cmd += ["-DNM_DBG_MODES"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-o", tmp, *sources()]

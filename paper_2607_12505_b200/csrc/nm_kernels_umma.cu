@@ -570,7 +570,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t sb = res_x ? slot : st;
           // metadata columns follow the copy of the metadata they hold: ring stage or K step
           const uint32_t meta_cols = tmem_meta + (res_w ? (uint32_t)ks : s) * 8u;
-#ifdef NM_TRACE
+#ifdef NM_HAS_DBG
           if (p.dbg & 1) { tc_commit(bar_empty + 8u * s); if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; st = ring_base; } else { st += sbytes; } continue; }
 #endif
           if (SP) {
@@ -651,7 +651,7 @@ nm_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int cc = (h ^ (n & 1)) * 32; cc < p.tile_t; cc += 64) {
         const int t = c.t0 + cc;
         if (t >= p.T) break;
-#ifdef NM_TRACE
+#ifdef NM_HAS_DBG
         if (p.dbg & 2) continue;
 #endif
         uint32_t r[32];
@@ -1038,7 +1038,7 @@ nm_status launch_umma(const SpmmArgs& a) {
   p.diag_stall = (pl.reserved & NM_PLAN_DIAG_STALL) ? 1 : 0;
   p.spin_limit = p.diag_stall ? (1u << 14) : kSpinLimit;
   p.trace = trace_buffer();
-#ifdef NM_TRACE
+#ifdef NM_HAS_DBG
   { const char* e = getenv("NM_DBG"); p.dbg = e ? atoi(e) : 0; }
 #endif
   if (dec) {

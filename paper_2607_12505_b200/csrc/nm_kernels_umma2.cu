@@ -189,7 +189,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int t0 = tile0 + (int)rank * (int)half_rows;
         if (p.T - tile0 < p.tile_t) t0 = tile0 + (int)rank * (((p.T - tile0 + 31) & ~31) >> 1);
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
-#ifdef NM_TRACE
+#ifdef NM_HAS_DBG
           if ((p.dbg & 4) && armed >= (uint32_t)p.stages) { n = my_count; break; }   // the ring is filled once and reused
 #endif
           if (wrapped) {
@@ -287,7 +287,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         t_idx += step_t; o_idx += step_o;
         if (o_idx >= p.tiles_o2) { o_idx -= p.tiles_o2; ++t_idx; }
         for (int ks = 0; ks < p.total_ksteps; ++ks) {
-#ifdef NM_TRACE
+#ifdef NM_HAS_DBG
           if (!((p.dbg & 4) && (n > 0 || ks >= p.stages)))      // 4 = no loads after the first ring-full: the MMAs run alone
 #endif
           NM_WAIT_TIMED(cyc_full, ok = mbar_wait(bar_full + 8u * s, ph, wctx, 2));
@@ -298,7 +298,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const uint32_t sm = sa + 16384u;
           const uint32_t sb = sm + meta_bytes2<DT, SP>();
           const uint32_t meta_cols = tmem_meta + s * 8u;
-#ifdef NM_TRACE
+#ifdef NM_HAS_DBG
           if (p.dbg & 1) { tc_commit_pair(bar_empty + 8u * s); if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1u; sa = smem_base; } else { sa += sbytes; } continue; }
 #endif
           if (SP) {
@@ -362,7 +362,7 @@ nm_umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int t = t0 + cc;
         if (t >= p.T) break;
         uint32_t r[32];
-#ifdef NM_TRACE
+#ifdef NM_HAS_DBG
         if (p.dbg & 2) continue;
 #endif
         if (lane == 0) tma_store_wait_read();
@@ -516,7 +516,7 @@ nm_status launch_umma_pair(const SpmmArgs& a, bool* handled) {
   p.status = a.status;
   p.spin_limit = kSpinLimit;
   p.trace = trace_buffer();
-#ifdef NM_TRACE
+#ifdef NM_HAS_DBG
   { const char* e = getenv("NM_DBG"); p.dbg = e ? atoi(e) : 0; }
 #endif
   p.w_fresh = a.w_fresh ? 1 : 0;

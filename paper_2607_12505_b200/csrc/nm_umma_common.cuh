@@ -48,6 +48,12 @@ __device__ __forceinline__ uint32_t requant_low_byte(uint32_t acc_bits, float sc
 // store issued, 9 staging patch free again, 10 about to free tensor memory, 12 tiles of this CTA;
 // SM cycles spent inside waits: 11 epilogue warp 2 for an accumulator, 13 issuing warp for a loaded
 // stage, 14 issuing warp for a drained accumulator, 15 producer for a free stage.
+// The timing experiments (NM_DBG: a GEMM without its MMAs, without its stores, over a ring loaded once) are
+// compiled into the trace build and into a third build, -DNM_DBG_MODES, that has them WITHOUT the stamp and
+// wait-timing code, whose cost in the inner loops is itself 20-30 % of a store-less run.
+#if defined(NM_TRACE) || defined(NM_DBG_MODES)
+#define NM_HAS_DBG 1
+#endif
 #ifdef NM_TRACE
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
