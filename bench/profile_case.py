@@ -7,6 +7,10 @@
 Prints one JSON line: microseconds per call (CUDA events on the launching stream, buffers
 rotated over `--rotate` sets so that consecutive calls do not hit L2), achieved GB/s on the
 algorithmic bytes (X once, Y once, packed W once) and dense-equivalent T(FL)OPS.
+
+With NM_B200_TRACE=2 in the environment the binding loads the timing build of the library
+(-DNM_DBG_MODES), in which NM_DBG switches parts of the tcgen05 kernels off at run time (bit 1: no
+MMAs, 2: no stores, 4: the ring is loaded once; results are then wrong by construction).
 """
 from __future__ import annotations
 

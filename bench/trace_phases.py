@@ -16,7 +16,8 @@ Timing experiments of the trace build (environment variable NM_DBG, read at laun
 warp issues no MMAs (stages are recycled at once), 2 = the epilogue stores nothing, 3 = both, i.e. only
 the operand loads run; 4 (CTA-pair kernel only) = the ring is loaded once and the K loops run over it
 without further loads, so 6 = the MMAs alone.  Results are wrong by construction; only the times mean
-something.
+something.  For timing these modes use `NM_B200_TRACE=2 python -m bench.profile_case ...`: that library
+has the switches without the stamp code, which slows the inner loops by itself.
 """
 from __future__ import annotations
 
